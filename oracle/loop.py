@@ -1,0 +1,96 @@
+"""CPU oracle for the decode loop (Algorithm 1) on synthetic hidden states -- TEST INFRASTRUCTURE.
+
+The transformer is replaced by the seeded generator: at every step the hidden states of the
+scored rows are re-drawn from (seed, step, sequence, position) with an amplitude that grows with
+the sequence's committed fraction.  Decoding is semi-autoregressive (Appendix A.1): the working
+block of a sequence is its first block that still holds a mask, and the scored rows are that
+block's masked positions.  One loop step = one batched forward (draft pass and verification
+branches counted together).
+
+`decode(..., budget=0)` is confidence-threshold decoding (Section 2): nothing is drafted, every
+step commits the base set only.
+"""
+from __future__ import annotations
+
+from typing import Dict
+
+import numpy as np
+
+from . import score as oscore
+from . import step as ostep
+
+
+def working_rows(y: np.ndarray, mask_id: int, block: int):
+    """Rows of the current step: for each unfinished sequence the masked positions of its first
+    block that holds a mask.  Returns seq_ids, positions (ascending per sequence), seg_off."""
+    n_seq, L = y.shape
+    seq_ids, positions = [], []
+    seg_off = np.zeros(n_seq + 1, dtype=np.int32)
+    for b in range(n_seq):
+        masked = np.nonzero(y[b] == mask_id)[0]
+        if len(masked):
+            k = int(masked[0]) // block
+            pos = [int(i) for i in masked if k * block <= i < (k + 1) * block]
+            seq_ids.extend([b] * len(pos))
+            positions.extend(pos)
+        seg_off[b + 1] = len(positions)
+    return np.asarray(seq_ids, np.int32), np.asarray(positions, np.int32), seg_off
+
+
+def decode(synth, w_bits, plan_ids, targets, seed: int, gen_len: int, block: int, params: Dict,
+           mask_id: int, max_steps: int = 100000, trace: bool = False) -> Dict:
+    """Run Algorithm 1 until no masks remain.  ``synth`` is the input-generator module."""
+    n_seq = targets.shape[0]
+    K = int(params["budget"])
+    y = np.full((n_seq, gen_len), mask_id, dtype=np.int32)
+    steps_per_seq = np.zeros(n_seq, dtype=np.int32)
+    scored_rows = 0
+    n_steps = 0
+    history = []
+    while (y == mask_id).any():
+        if n_steps >= max_steps:
+            raise RuntimeError("decode loop did not terminate")
+        seq_ids, positions, seg_off = working_rows(y, mask_id, block)
+        frac = (y != mask_id).sum(axis=1) / float(gen_len)
+        h = synth.loop_hidden(w_bits, targets, seed, n_steps, 0, seq_ids, positions, frac)
+        sc = oscore.score(w_bits, h, plan_ids)
+        active = np.ones(len(positions), np.uint8)
+        cm = ostep.commit(sc["conf"], sc["tok"], seg_off, positions, active, params["tau_high"],
+                          force_progress=True)
+        scored_rows += len(positions)
+        final = cm["commit"]
+        sel = ver = None
+        if K > 0:
+            sel = ostep.select_drafts(sc["conf"], sc["tok"], sc["in_plan"], cm["commit"], seg_off,
+                                      positions, active, params["tau_plan_lo"], params["tau_plan_hi"],
+                                      params["tau_ar_lo"], K)
+            vb, vi, vc = [], [], []
+            for b in range(n_seq):
+                rem = sel["rem_rows"][sel["rem_off"][b]:sel["rem_off"][b + 1]]
+                if sel["n_drafts"][b] > 0:
+                    for c in range(1 + int(sel["n_drafts"][b])):
+                        for m in rem:
+                            vb.append(b); vi.append(int(positions[m])); vc.append(c)
+            hv = synth.loop_verify_hidden(w_bits, targets, seed, n_steps, np.asarray(vb, np.int32),
+                                          np.asarray(vi, np.int32), np.asarray(vc, np.int32), frac)
+            scv = oscore.score(w_bits, hv, plan_ids)
+            scored_rows += len(vb)
+            ver = ostep.verify(sc["tok"], cm["commit"], seg_off, positions, sel["rem_rows"],
+                               sel["rem_off"], sel["v_off"], sel["draft_rows"], sel["n_drafts"],
+                               sel["route"], scv["tok"], scv["conf"], params["tau_high"], K)
+            final = ver["final_commit"]
+        for m in range(len(positions)):
+            if final[m]:
+                y[seq_ids[m], positions[m]] = sc["tok"][m]
+        for b in range(n_seq):
+            if seg_off[b + 1] > seg_off[b]:
+                steps_per_seq[b] += 1
+        if trace:
+            history.append(dict(positions=positions.copy(), seq_ids=seq_ids.copy(), score=sc,
+                                commit=cm, select=sel, verify=ver, y=y.copy()))
+        n_steps += 1
+    out = dict(y=y, steps=n_steps, steps_per_seq=steps_per_seq, scored_rows=scored_rows,
+               tokens_per_forward=float(np.mean(gen_len / np.maximum(steps_per_seq, 1))))
+    if trace:
+        out["history"] = history
+    return out
