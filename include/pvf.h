@@ -1,0 +1,189 @@
+/*
+ * pvf.h -- C interface of the B200 (sm_100a) Plan-Verify-Fill vocabulary pass.
+ *
+ * One decode step of PVF (Algorithm 1 of the paper) as four device-side calls:
+ *
+ *   pvf_score          hidden states of the masked positions -> top-1 token, confidence, entropy,
+ *                      planning-vocabulary membership (LM-head GEMM fused with a streaming softmax;
+ *                      logits never reach global memory)
+ *   pvf_commit         confidence-threshold base set S_base and base branch z_base
+ *   pvf_select_drafts  planning candidates P_t^plan -> top-K drafts, else the AR fallback list
+ *   pvf_verify         impact-set acceptance A_t^j, branch choice by C_total, AR k*, final commit
+ *
+ * Conventions common to all calls
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless it is marked "host".  The
+ *     library never frees caller memory and keeps no pointer beyond a call, except the LM-head
+ *     weight and the workspace handed to pvf_create, which must outlive the context.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = the legacy default
+ *     stream); they never synchronise and never read device results on the host.
+ *   - Return value: PVF_OK or a negative PVF_ERR_* code.  On an argument error nothing is launched.
+ *     Nothing is printed, thrown or aborted.
+ *   - Kernels bound every internal wait; a wait that runs out stores PVF_ERR_TIMEOUT in the
+ *     context's device status word (read it with pvf_last_status after synchronising).
+ *   - Token ids, positions and row indices are int32; masks and flags uint8 (0/1); confidences and
+ *     entropies float32; hidden states and weights bf16 (the usual 16-bit layout), row-major.
+ *   - Rows.  The M scored rows ("masked positions") are grouped by sequence: rows of sequence b are
+ *     seg_off[b] .. seg_off[b+1]-1 (seg_off has n_seq+1 entries, seg_off[0] = 0, seg_off[n_seq] = M),
+ *     sorted by ascending canvas position row_pos[m].  active[m] != 0 says the position belongs to the
+ *     working block B_t (NULL = every row is active).  M = 0 and n_seq = 0 are valid no-ops.
+ *   - Calls on one context share its workspace: they must not overlap on the GPU (use one stream, or
+ *     order them with events).  Different contexts are independent.
+ *   - There is no CPU fallback: every call needs a device of compute capability 10.0.
+ */
+#ifndef PVF_H_
+#define PVF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct pvf_ctx pvf_ctx;
+
+enum {
+    PVF_OK = 0,
+    PVF_ERR_INVALID = -1,     /* NULL required pointer, negative size, size above the context's limits */
+    PVF_ERR_ALIGN = -2,       /* weight / hidden pointer not 16-byte aligned, hidden size not a multiple of 8 */
+    PVF_ERR_UNSUPPORTED = -3, /* device is not sm_100, or a shape outside what the kernels handle */
+    PVF_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed */
+    PVF_ERR_TIMEOUT = -5,     /* (status word only) a bounded wait inside a kernel ran out */
+    PVF_ERR_WORKSPACE = -6    /* workspace too small or not 256-byte aligned */
+};
+
+/* Limits of a context.  max_rows bounds M of every call, max_seqs bounds n_seq, max_budget bounds K. */
+typedef struct {
+    int32_t vocab;      /* V: rows of the LM-head weight */
+    int32_t hidden;     /* D: multiple of 8 */
+    int32_t max_rows;
+    int32_t max_seqs;
+    int32_t max_budget;
+} pvf_shape;
+
+#define PVF_FORCE_PROGRESS            1u  /* a sequence with active rows but an empty base set commits its
+                                             single most confident active row (lowest position on ties) */
+#define PVF_EXCLUDE_SELF_FROM_IMPACT  2u  /* leave draft j's own position out of the impact set of branch j */
+
+/* Thresholds of the step.  Names follow the paper: tau_high (Section 2), the planning band
+ * [tau_plan_lo, tau_plan_hi) (Section 4.1), tau_ar_lo (Section 4.3), budget = K drafts per sequence. */
+typedef struct {
+    float    tau_high;
+    float    tau_plan_lo;
+    float    tau_plan_hi;
+    float    tau_ar_lo;
+    int32_t  budget;
+    uint32_t flags;
+} pvf_params;
+
+/* The paper's printed defaults: tau_high = 0.9, K = 3 (Section 5.1); planning band (0.2, 0.65) and
+ * tau_AR^l = 0.1 (Table 5, GSM8K / MMLU-Pro rows); flags = 0. */
+void pvf_default_params(pvf_params *out);
+
+const char *pvf_strerror(int code);
+
+/* Bytes of device workspace a context of this shape needs (0 on an invalid shape).  Needs a
+ * current CUDA device (the layout depends on its SM count). */
+size_t pvf_workspace_bytes(const pvf_shape *shape);
+
+/*
+ * Create a context.
+ *   w_head          device, bf16 [vocab][hidden] row-major, 16-byte aligned: the LM head.  Kept.
+ *   plan_ids_host   HOST, n_plan token ids of the planning vocabulary P^plan (Section 3; any order,
+ *                   duplicates allowed, each in [0, vocab)).  Copied into a device bitmap during the
+ *                   call (this call synchronises the device once).
+ *   workspace       device, >= pvf_workspace_bytes(shape) bytes, 256-byte aligned.  Kept.
+ * The context belongs to the CUDA device that is current during the call.
+ */
+int pvf_create(pvf_ctx **out, const pvf_shape *shape, const void *w_head,
+               const int32_t *plan_ids_host, int32_t n_plan, void *workspace, size_t workspace_bytes);
+int pvf_destroy(pvf_ctx *ctx);
+
+/* Copies the device status word to *status (PVF_OK or PVF_ERR_TIMEOUT) and clears it.
+ * Synchronises the device. */
+int pvf_last_status(pvf_ctx *ctx, int32_t *status);
+
+/*
+ * Launch geometry pvf_score would use for M rows; any pointer may be NULL.
+ *   ctas        thread blocks of the GEMM kernel            splits   vocabulary ranges per row tile
+ *   waves       passes over the weight matrix               launches kernels launched per call
+ */
+int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int32_t *waves, int32_t *launches);
+
+/*
+ * pvf_score -- the vocabulary pass of one forward (Section 2 "confidence-based parallel decoding";
+ * Section 3, definitions of y^_t^i, p_t^i and H_i; Section 4.1, "y^ in P^plan").
+ *
+ *   hidden   [M][hidden] bf16, 16-byte aligned: final hidden state of each scored position.
+ * For each row m with logits x_v = sum_k hidden[m][k] * w_head[v][k] (bf16 products, fp32 accumulation)
+ * and q = softmax(x):
+ *   tok[m]     = argmax_v x_v, the lowest id on ties            conf[m] = q[tok[m]]
+ *   ent[m]     = -sum_v q_v ln q_v  (nats)                      in_plan[m] = tok[m] in P^plan
+ * ent and in_plan may be NULL.  Non-finite hidden values leave that row's outputs unspecified;
+ * the call still terminates and stays in bounds.
+ */
+int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
+              int32_t *tok, float *conf, float *ent, uint8_t *in_plan, void *stream);
+
+/*
+ * pvf_commit -- base set and base branch (Section 2, threshold rule; Section 3, S_base and z_base).
+ *   commit[m]   = active[m] && conf[m] >= tau_high     (plus the forced row, see PVF_FORCE_PROGRESS)
+ *   n_commit[b] = committed rows of sequence b                                   (may be NULL)
+ *   y           canvas [n_seq][L] in/out or NULL: y[b][row_pos[m]] = tok[m] at committed rows, every
+ *               other entry untouched (committed positions are never re-masked).
+ */
+int pvf_commit(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
+               const int32_t *seg_off, const int32_t *row_pos, const uint8_t *active,
+               const int32_t *tok, const float *conf,
+               uint8_t *commit, int32_t *n_commit, int32_t *y, int32_t L, void *stream);
+
+/*
+ * pvf_select_drafts -- draft proposal (Section 4.1 planning candidates and TopK; Section 4.3 AR
+ * candidate construction; Algorithm 1, route switch).
+ * Per sequence b, with R_b = its rows that are active and not in `commit`, in position order:
+ *   planning candidates = rows of R_b with in_plan != 0 and tau_plan_lo <= conf < tau_plan_hi;
+ *   if there are any (and budget > 0): the K_t = min(budget, count) most confident, ties to the lower
+ *     position, written in rank order; route = 1.
+ *   otherwise: the first <= budget rows of R_b with conf >= tau_ar_lo, in position order; route = 2,
+ *     or route = 0 when there is none.
+ * Outputs
+ *   draft_rows [n_seq][budget]  row indices, -1 padded         n_drafts [n_seq]
+ *   route      [n_seq]          0 none, 1 planning, 2 AR
+ *   rem_rows   [<= M]           R_b of every sequence, concatenated   rem_off [n_seq+1]
+ *   v_off      [n_seq+1]        row offsets of the verification pass: sequence b owns
+ *                               (1 + n_drafts[b]) * |R_b| rows if it has drafts, else none.
+ */
+int pvf_select_drafts(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
+                      const int32_t *seg_off, const int32_t *row_pos, const uint8_t *active,
+                      const int32_t *tok, const float *conf, const uint8_t *in_plan,
+                      const uint8_t *commit,
+                      int32_t *draft_rows, int32_t *n_drafts, uint8_t *route,
+                      int32_t *rem_rows, int32_t *rem_off, int32_t *v_off, void *stream);
+
+/*
+ * pvf_verify -- acceptance check and final commit (Eq. 1 impact set, Eq. 3 verified compatibility,
+ * Section 4.2 Filter 1 and Filter 2, Section 4.3 AR verification and selection).
+ *   tok_v, conf_v   pvf_score outputs of the verification pass, rows [b][c][r]: index
+ *                   v_off[b] + c * |R_b| + r; c = 0 is the base branch, c = j the branch that adds draft
+ *                   j (planning) or the first j fills (AR); r indexes rem_rows of sequence b.
+ *   tok             tokens of the draft pass (the drafted tokens).
+ * Planning route: S_impact = {r : conf_v[base][r] >= tau_high}; accept[b][j-1] = S_impact non-empty and
+ *   tok_v[j][r] == tok_v[base][r] on all of it; C_j = sum over r != draft j of conf_v[j][r] (fp64, in row
+ *   order); choice[b] = the accepted j with the largest C_j (lowest j on ties), 0 if none.
+ * AR route: accept[b][k-1] = for all r <= k: tok_v[k][row of fill r] == tok[fill r];
+ *   choice[b] = largest accepted k, 0 if none.
+ * final_commit = commit, plus draft `choice` (planning) or fills 1..choice (AR).  y as in pvf_commit,
+ * written at every final_commit row.  accept entries beyond n_drafts[b] are 0.
+ */
+int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
+               const int32_t *seg_off, const int32_t *row_pos,
+               const int32_t *rem_rows, const int32_t *rem_off, const int32_t *v_off,
+               const int32_t *draft_rows, const int32_t *n_drafts, const uint8_t *route,
+               const int32_t *tok, const int32_t *tok_v, const float *conf_v, const uint8_t *commit,
+               uint8_t *accept, int32_t *choice, uint8_t *final_commit,
+               int32_t *y, int32_t L, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PVF_H_ */

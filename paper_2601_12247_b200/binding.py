@@ -1,0 +1,207 @@
+"""Thin ctypes binding of libpvf.so: argument marshalling only.
+
+Every function here has the name and meaning of the C entry point it calls (see include/pvf.h);
+torch is used for device memory and for the current stream, nothing else.  There is no fallback:
+if the library has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpvf.so")
+
+PVF_OK = 0
+PVF_ERR_INVALID, PVF_ERR_ALIGN, PVF_ERR_UNSUPPORTED, PVF_ERR_CUDA, PVF_ERR_TIMEOUT, PVF_ERR_WORKSPACE = -1, -2, -3, -4, -5, -6
+PVF_FORCE_PROGRESS = 1
+PVF_EXCLUDE_SELF_FROM_IMPACT = 2
+
+
+class pvf_shape(ctypes.Structure):
+    _fields_ = [("vocab", ctypes.c_int32), ("hidden", ctypes.c_int32), ("max_rows", ctypes.c_int32),
+                ("max_seqs", ctypes.c_int32), ("max_budget", ctypes.c_int32)]
+
+
+class pvf_params(ctypes.Structure):
+    _fields_ = [("tau_high", ctypes.c_float), ("tau_plan_lo", ctypes.c_float), ("tau_plan_hi", ctypes.c_float),
+                ("tau_ar_lo", ctypes.c_float), ("budget", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class PvfError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        super().__init__("%s failed: %d (%s)" % (what, code, strerror(code)))
+        self.code = code
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libpvf.so; raises if it is missing (build it with paper_2601_12247_b200/build.py)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libpvf.so is not built: run `python -m paper_2601_12247_b200.build` "
+                               "(there is no CPU or PyTorch fallback)")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        pp = ctypes.POINTER(pvf_params)
+        ps = ctypes.POINTER(pvf_shape)
+        lib.pvf_default_params.argtypes = [pp]; lib.pvf_default_params.restype = None
+        lib.pvf_strerror.argtypes = [ctypes.c_int]; lib.pvf_strerror.restype = ctypes.c_char_p
+        lib.pvf_workspace_bytes.argtypes = [ps]; lib.pvf_workspace_bytes.restype = sz
+        lib.pvf_create.argtypes = [ctypes.POINTER(vp), ps, vp, vp, i32, vp, sz]; lib.pvf_create.restype = ctypes.c_int
+        lib.pvf_destroy.argtypes = [vp]; lib.pvf_destroy.restype = ctypes.c_int
+        lib.pvf_last_status.argtypes = [vp, ctypes.POINTER(i32)]; lib.pvf_last_status.restype = ctypes.c_int
+        lib.pvf_score_plan.argtypes = [vp, i32] + [ctypes.POINTER(i32)] * 4; lib.pvf_score_plan.restype = ctypes.c_int
+        lib.pvf_score.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]; lib.pvf_score.restype = ctypes.c_int
+        lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
+        lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
+        lib.pvf_verify.argtypes = [vp, pp, i32, i32] + [vp] * 16 + [i32, vp]; lib.pvf_verify.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return load().pvf_strerror(int(code)).decode()
+
+
+def default_params() -> pvf_params:
+    p = pvf_params()
+    load().pvf_default_params(ctypes.byref(p))
+    return p
+
+
+def make_params(tau_high: float, tau_plan_lo: float, tau_plan_hi: float, tau_ar_lo: float, budget: int,
+                flags: int = 0) -> pvf_params:
+    return pvf_params(tau_high, tau_plan_lo, tau_plan_hi, tau_ar_lo, int(budget), int(flags))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc: int, what: str):
+    if rc != PVF_OK:
+        raise PvfError(rc, what)
+
+
+class Context:
+    """Owns a pvf_ctx, its workspace and a reference to the LM-head weight."""
+
+    def __init__(self, w_head: torch.Tensor, plan_ids, max_rows: int, max_seqs: int, max_budget: int):
+        lib = load()
+        assert w_head.is_cuda and w_head.dtype == torch.bfloat16 and w_head.is_contiguous() and w_head.dim() == 2
+        self.lib = lib
+        self.w_head = w_head
+        self.device = w_head.device
+        self.shape = pvf_shape(w_head.shape[0], w_head.shape[1], int(max_rows), int(max_seqs), int(max_budget))
+        with torch.cuda.device(self.device):
+            nbytes = lib.pvf_workspace_bytes(ctypes.byref(self.shape))
+            if nbytes == 0:
+                raise PvfError(PVF_ERR_INVALID, "pvf_workspace_bytes")
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            off = (-self.workspace.data_ptr()) % 256
+            ids = np.ascontiguousarray(np.asarray(plan_ids, dtype=np.int32))
+            self.handle = ctypes.c_void_p()
+            rc = lib.pvf_create(ctypes.byref(self.handle), ctypes.byref(self.shape), _ptr(w_head),
+                                ids.ctypes.data_as(ctypes.c_void_p), len(ids),
+                                ctypes.c_void_p(self.workspace.data_ptr() + off), nbytes)
+        _check(rc, "pvf_create")
+
+    def close(self):
+        if getattr(self, "handle", None) is not None and self.handle.value:
+            self.lib.pvf_destroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def last_status(self) -> int:
+        st = ctypes.c_int32()
+        _check(self.lib.pvf_last_status(self.handle, ctypes.byref(st)), "pvf_last_status")
+        return int(st.value)
+
+    def score_plan(self, M: int) -> Dict[str, int]:
+        v = [ctypes.c_int32() for _ in range(4)]
+        _check(self.lib.pvf_score_plan(self.handle, int(M), *[ctypes.byref(x) for x in v]), "pvf_score_plan")
+        return dict(ctas=v[0].value, splits=v[1].value, waves=v[2].value, launches=v[3].value)
+
+    # ------------------------------------------------------------------ the four calls
+    def score(self, hidden: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
+        assert hidden.is_cuda and hidden.dtype == torch.bfloat16 and hidden.is_contiguous()
+        M = hidden.shape[0]
+        if out is None:
+            out = dict(tok=torch.empty(M, dtype=torch.int32, device=self.device),
+                       conf=torch.empty(M, dtype=torch.float32, device=self.device),
+                       ent=torch.empty(M, dtype=torch.float32, device=self.device),
+                       in_plan=torch.empty(M, dtype=torch.uint8, device=self.device))
+        rc = self.lib.pvf_score(self.handle, _ptr(hidden), M, _ptr(out["tok"]), _ptr(out["conf"]),
+                                _ptr(out.get("ent")), _ptr(out.get("in_plan")), _stream())
+        _check(rc, "pvf_score")
+        return out
+
+    def commit(self, params: pvf_params, seg_off, row_pos, active, tok, conf, y=None, out=None):
+        M, n_seq = conf.shape[0], seg_off.shape[0] - 1
+        if out is None:
+            out = dict(commit=torch.empty(M, dtype=torch.uint8, device=self.device),
+                       n_commit=torch.empty(n_seq, dtype=torch.int32, device=self.device))
+        L = 0 if y is None else y.shape[1]
+        rc = self.lib.pvf_commit(self.handle, ctypes.byref(params), M, n_seq, _ptr(seg_off), _ptr(row_pos),
+                                 _ptr(active), _ptr(tok), _ptr(conf), _ptr(out["commit"]), _ptr(out["n_commit"]),
+                                 _ptr(y), L, _stream())
+        _check(rc, "pvf_commit")
+        return out
+
+    def select_drafts(self, params: pvf_params, seg_off, row_pos, active, tok, conf, in_plan, commit, out=None):
+        M, n_seq, K = conf.shape[0], seg_off.shape[0] - 1, int(params.budget)
+        if out is None:
+            dev = self.device
+            out = dict(draft_rows=torch.empty((n_seq, K), dtype=torch.int32, device=dev),
+                       n_drafts=torch.empty(n_seq, dtype=torch.int32, device=dev),
+                       route=torch.empty(n_seq, dtype=torch.uint8, device=dev),
+                       rem_rows=torch.empty(max(M, 1), dtype=torch.int32, device=dev),
+                       rem_off=torch.empty(n_seq + 1, dtype=torch.int32, device=dev),
+                       v_off=torch.empty(n_seq + 1, dtype=torch.int32, device=dev))
+        rc = self.lib.pvf_select_drafts(self.handle, ctypes.byref(params), M, n_seq, _ptr(seg_off), _ptr(row_pos),
+                                        _ptr(active), _ptr(tok), _ptr(conf), _ptr(in_plan), _ptr(commit),
+                                        _ptr(out["draft_rows"]), _ptr(out["n_drafts"]), _ptr(out["route"]),
+                                        _ptr(out["rem_rows"]), _ptr(out["rem_off"]), _ptr(out["v_off"]), _stream())
+        _check(rc, "pvf_select_drafts")
+        return out
+
+    def verify(self, params: pvf_params, seg_off, row_pos, sel: Dict[str, torch.Tensor], tok, tok_v, conf_v,
+               commit, y=None, out=None):
+        M, n_seq, K = commit.shape[0], seg_off.shape[0] - 1, int(params.budget)
+        if out is None:
+            dev = self.device
+            out = dict(accept=torch.empty((n_seq, K), dtype=torch.uint8, device=dev),
+                       choice=torch.empty(n_seq, dtype=torch.int32, device=dev),
+                       final_commit=torch.empty(M, dtype=torch.uint8, device=dev))
+        L = 0 if y is None else y.shape[1]
+        rc = self.lib.pvf_verify(self.handle, ctypes.byref(params), M, n_seq, _ptr(seg_off), _ptr(row_pos),
+                                 _ptr(sel["rem_rows"]), _ptr(sel["rem_off"]), _ptr(sel["v_off"]),
+                                 _ptr(sel["draft_rows"]), _ptr(sel["n_drafts"]), _ptr(sel["route"]),
+                                 _ptr(tok), _ptr(tok_v), _ptr(conf_v), _ptr(commit),
+                                 _ptr(out["accept"]), _ptr(out["choice"]), _ptr(out["final_commit"]),
+                                 _ptr(y), L, _stream())
+        _check(rc, "pvf_verify")
+        return out
+
+
+def bf16_from_bits(bits: np.ndarray, device) -> torch.Tensor:
+    """uint16 bf16 bit patterns (numpy) -> torch.bfloat16 tensor on `device`."""
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)

@@ -1,0 +1,51 @@
+// Internal declarations shared by the translation units of libpvf (not part of the C interface).
+#ifndef PVF_INTERNAL_H_
+#define PVF_INTERNAL_H_
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "pvf.h"
+
+#define PVF_MAX_BUDGET_LIMIT 64
+
+// Device scalars at the head of the workspace.
+struct pvf_device_words {
+    int32_t  status;        // PVF_OK or PVF_ERR_TIMEOUT, written by kernels
+    uint32_t select_ticket; // blocks of pvf_select_drafts that have finished; reset by the last one
+    uint32_t pad[62];
+};
+
+struct pvf_ctx {
+    pvf_shape shape;
+    int device;
+    int n_sm;
+    const void *w_head;
+    uint8_t *workspace;
+    size_t workspace_bytes;
+    pvf_device_words *words;
+    uint32_t *plan_bitmap;  // ceil(V/32) words, bit v set iff v in P^plan
+    float4 *partials;       // [rows][splits] per-range softmax states of pvf_score
+    size_t partials_bytes;
+    CUtensorMap tm_w_full;  // W as [V][D], box 256 rows x 64 columns, 128-byte swizzle
+    CUtensorMap tm_w_unit;  // same tensor, box 16 rows x 64 columns
+};
+
+// Work split of pvf_score for M rows on n_sm SMs (see pvf_score.cu).
+struct pvf_score_geometry {
+    int m_tiles;     // ceil(M / 128)
+    int units;       // ceil(V / 16): vocabulary granules
+    int mb;          // row tiles processed concurrently (one wave)
+    int splits;      // vocabulary ranges per row tile = partial states per row
+    int waves;       // ceil(m_tiles / mb)
+    int ctas;        // mb * splits
+    int a_rows;      // rows of the hidden-state TMA box
+};
+pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm);
+size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm);
+int pvf_score_init(pvf_ctx *ctx);   // tensor maps of W, kernel attributes
+
+static inline size_t pvf_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+#endif

@@ -1,0 +1,601 @@
+// pvf_score: LM-head projection fused with a streaming softmax (sm_100a).
+//
+//   logits[m][v] = sum_k H[m][k] * W[v][k]      bf16 operands, fp32 accumulation in tensor memory
+//   per row m:     top-1 token, its probability, the entropy of softmax(logits[m][:])
+//
+// The logits never leave the SM.  Scored rows sit on the 128 lanes of a tcgen05 accumulator, the
+// vocabulary on its columns, so one epilogue thread owns one row and keeps that row's running
+// softmax state (max, argmax, sum e^{x-max}, sum (x-max) e^{x-max}) in registers while the thread
+// block sweeps a contiguous vocabulary range.  Each (row, range) pair leaves one 16-byte partial
+// state; a small second kernel merges the partials of a row.
+//
+// Thread block = 6 warps:  warp 0 issues TMA loads (W and H tiles, 128-byte swizzle, 4 stages),
+// warp 1 owns tensor memory and issues the MMAs, warps 2-5 are the softmax epilogue.  The two
+// 256-column accumulators alternate, so the epilogue of one vocabulary tile overlaps the MMAs of
+// the next.
+//
+// Work split.  Rows form tiles of 128, the vocabulary granules of 16 entries.  `mb` row tiles are
+// in flight at once, each swept by `splits` blocks over disjoint vocabulary ranges (mb * splits
+// <= number of SMs); blocks that share a range stream the same W tiles at the same time, so W is
+// read from HBM once per wave, and the wave's H tiles stay L2-resident.
+//   M <= 128:  one row tile, one range per SM (pure weight streaming)
+//   M large:   waves of up to 64 row tiles
+//
+// Every wait on an mbarrier is bounded: when one runs out the block records PVF_ERR_TIMEOUT in
+// the status word, raises a block-wide abort flag, drains its outstanding copies and MMAs with
+// bounded waits, frees its tensor memory and returns.
+#include <math.h>
+
+#include "pvf_internal.h"
+
+namespace {
+
+constexpr int kTileM = 128;                // rows per accumulator (tensor-memory lanes)
+constexpr int kTileN = 256;                // vocabulary entries per accumulator (columns)
+constexpr int kUnit = 16;                  // vocabulary granule
+constexpr int kBlockK = 64;                // bf16 per k-block = one 128-byte swizzle row
+constexpr int kStages = 4;
+constexpr int kABytes = kTileM * kBlockK * 2;          // 16 KiB
+constexpr int kBBytes = kTileN * kBlockK * 2;          // 32 KiB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kUnitBytes = kUnit * kBlockK * 2;        // 2 KiB
+constexpr int kThreads = 192;
+constexpr int kEpilogueThreads = 128;
+constexpr int kTmemCols = 512;
+constexpr int kMaxConcurrentTiles = 64;    // cap on the wave's L2-resident H tiles
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct __align__(8) SharedControl {
+    unsigned long long full[kStages];      // TMA bytes landed
+    unsigned long long empty[kStages];     // MMAs that read the stage have completed
+    unsigned long long acc_full[2];        // accumulator complete
+    unsigned long long acc_empty[2];       // epilogue has drained the accumulator
+    unsigned long long drain;              // abort path: all issued MMAs completed
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*control*/;
+
+struct ScoreArgs {
+    int M, V, D;
+    int num_kb;          // ceil(D / 64)
+    int units;           // ceil(V / 16)
+    int m_tiles, mb, splits, waves;
+    int a_rows;          // rows per H box
+    float4 *partials;    // [M][splits]
+    int32_t *status;
+};
+
+// ---------------------------------------------------------------------------------- PTX helpers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false when the block is aborting (this wait ran out, or another did).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, SharedControl *ctl, int32_t *status)
+{
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (ctl->abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) {
+            ctl->abort_flag = 1;
+            atomicExch(status, (int32_t)PVF_ERR_TIMEOUT);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, SharedControl *ctl, int32_t *status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, ctl, status);
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, one 128 x N x 16 bf16 MMA.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) with the
+// 128-byte swizzle: 8-row groups are 1024 bytes apart (stride offset), the leading offset is unused.
+__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);         // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                          // leading byte offset (ignored for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset
+    d |= (uint64_t)1 << 46;                          // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;                          // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+#define PVF_TMEM_LD_ARGS(v, o) \
+    "=r"(v[o + 0]), "=r"(v[o + 1]), "=r"(v[o + 2]), "=r"(v[o + 3]), "=r"(v[o + 4]), "=r"(v[o + 5]), \
+    "=r"(v[o + 6]), "=r"(v[o + 7]), "=r"(v[o + 8]), "=r"(v[o + 9]), "=r"(v[o + 10]), "=r"(v[o + 11]), \
+    "=r"(v[o + 12]), "=r"(v[o + 13]), "=r"(v[o + 14]), "=r"(v[o + 15])
+
+// 16 consecutive fp32 columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : PVF_TMEM_LD_ARGS(v, 0) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ---------------------------------------------------------------------------------- work split
+// Vocabulary granules [u0, u1) of split q.
+__device__ __forceinline__ void split_range(int units, int splits, int q, int *u0, int *u1)
+{
+    *u0 = (int)((long long)units * q / splits);
+    *u1 = (int)((long long)units * (q + 1) / splits);
+}
+
+// Running softmax state of one row over the columns seen so far.
+struct RowState {
+    float m;      // running max
+    float s;      // sum e^{x - m}
+    float t;      // sum (x - m) e^{x - m}
+    int arg;      // lowest id attaining m
+};
+
+// Folds 16 logits (ids col0 .. col0+15; only the first n are real when !kFull) into the state.
+template <bool kFull>
+__device__ __forceinline__ void fold16(RowState &st, const uint32_t (&raw)[16], int col0, int n)
+{
+    constexpr float kLog2e = 1.4426950408889634f;
+    float x[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) x[i] = (kFull || i < n) ? __uint_as_float(raw[i]) : -INFINITY;
+    float cm = x[0];
+#pragma unroll
+    for (int i = 1; i < 16; ++i) cm = fmaxf(cm, x[i]);
+    if (cm > st.m) {                                   // strict: an equal later logit keeps the lower id
+        int idx = 15;
+#pragma unroll
+        for (int i = 14; i >= 0; --i) idx = (x[i] == cm) ? i : idx;
+        const float d = st.m - cm;                     // -inf on the first fold: the state is empty then
+        const float c = (st.s > 0.f) ? fast_exp2(d * kLog2e) : 0.f;
+        st.t = (st.s > 0.f) ? (st.t + d * st.s) * c : 0.f;
+        st.s *= c;
+        st.m = cm;
+        st.arg = col0 + idx;
+    }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        if (kFull || i < n) {
+            const float d = x[i] - st.m;
+            const float e = fast_exp2(d * kLog2e);
+            st.s += e;
+            st.t = fmaf(d, e, st.t);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------- GEMM kernel
+__global__ void __launch_bounds__(kThreads, 1)
+pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w_full,
+                      const __grid_constant__ CUtensorMap tm_w_unit, const ScoreArgs args)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
+    uint8_t *tiles_ptr = smem_raw + (tiles_addr - raw_addr);
+    SharedControl *ctl = reinterpret_cast<SharedControl *>(tiles_ptr + kStages * kStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int mt_local = blockIdx.x % args.mb;
+    const int q = blockIdx.x / args.mb;
+    int u0, u1;
+    split_range(args.units, args.splits, q, &u0, &u1);
+    const int n_tiles = (u1 - u0 + (kTileN / kUnit) - 1) / (kTileN / kUnit);   // vocabulary tiles per sweep
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueThreads);
+        }
+        mbar_init(smem_u32(&ctl->drain), 1);
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctl->tmem_base)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w_full) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w_unit) : "memory");
+            int stage = 0;
+            uint32_t phase = 0;
+            int armed_parity[kStages];
+#pragma unroll
+            for (int s = 0; s < kStages; ++s) armed_parity[s] = -1;
+            bool alive = true;
+            for (int w = 0; w < args.waves && alive; ++w) {
+                const int m_tile = w * args.mb + mt_local;
+                if (m_tile >= args.m_tiles) continue;
+                for (int tile = 0; tile < n_tiles && alive; ++tile) {
+                    const int tu0 = u0 + tile * (kTileN / kUnit);
+                    const int tun = min(kTileN / kUnit, u1 - tu0);              // granules in this tile
+                    const uint32_t bytes = (uint32_t)args.a_rows * (kBlockK * 2) + (uint32_t)tun * kUnitBytes;
+                    for (int kb = 0; kb < args.num_kb; ++kb) {
+                        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                        const uint32_t full = smem_u32(&ctl->full[stage]);
+                        const uint32_t a_dst = tiles_addr + stage * kStageBytes;
+                        const uint32_t b_dst = a_dst + kABytes;
+                        mbar_arrive_expect_tx(full, bytes);
+                        armed_parity[stage] = (int)phase;
+                        tma_load_2d(a_dst, &tm_h, full, kb * kBlockK, m_tile * kTileM);
+                        if (tun == kTileN / kUnit) {
+                            tma_load_2d(b_dst, &tm_w_full, full, kb * kBlockK, tu0 * kUnit);
+                        } else {
+                            for (int u = 0; u < tun; ++u)
+                                tma_load_2d(b_dst + u * kUnitBytes, &tm_w_unit, full, kb * kBlockK, (tu0 + u) * kUnit);
+                        }
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!alive) {
+                // Abort: let every copy this thread started land before the block's memory is released.
+                for (int s = 0; s < kStages; ++s)
+                    if (armed_parity[s] >= 0) {
+                        const unsigned long long t0 = global_timer_ns();
+                        while (!mbar_try_wait(smem_u32(&ctl->full[s]), (uint32_t)armed_parity[s]) &&
+                               global_timer_ns() - t0 < kWaitLimitNs) {}
+                    }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t tile_count = 0;
+            bool alive = true;
+            for (int w = 0; w < args.waves && alive; ++w) {
+                const int m_tile = w * args.mb + mt_local;
+                if (m_tile >= args.m_tiles) continue;
+                for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
+                    const int tu0 = u0 + tile * (kTileN / kUnit);
+                    const int tun = min(kTileN / kUnit, u1 - tu0);
+                    const uint32_t idesc = instr_desc_bf16(tun * kUnit);
+                    const uint32_t buf = tile_count & 1u;
+                    const uint32_t acc_phase = (tile_count >> 1) & 1u;
+                    if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), acc_phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t tmem_d = tmem_base + buf * kTileN;
+                    for (int kb = 0; kb < args.num_kb; ++kb) {
+                        if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, ctl, args.status)) { alive = false; break; }
+                        tc_fence_after_sync();
+                        const uint32_t a_addr = tiles_addr + stage * kStageBytes;
+                        const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
+                        const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kBlockK / 16; ++k)       // 16 bf16 = 32 bytes further along K
+                            tc_mma_bf16(tmem_d, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc,
+                                        (kb | k) != 0 ? 1u : 0u);
+                        tc_commit(smem_u32(&ctl->empty[stage]));
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (alive) tc_commit(smem_u32(&ctl->acc_full[buf]));
+                }
+            }
+            if (!alive) {
+                // Abort: wait (bounded) until every MMA issued so far has retired.
+                tc_commit(smem_u32(&ctl->drain));
+                const unsigned long long t0 = global_timer_ns();
+                while (!mbar_try_wait(smem_u32(&ctl->drain), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax epilogue
+        const int quad = warp & 3;                               // tensor-memory lanes quad*32 .. quad*32+31
+        const int row_in_tile = quad * 32 + lane;
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        uint32_t tile_count = 0;
+        bool alive = true;
+        for (int w = 0; w < args.waves && alive; ++w) {
+            const int m_tile = w * args.mb + mt_local;
+            if (m_tile >= args.m_tiles) continue;
+            const int row = m_tile * kTileM + row_in_tile;
+            const bool warp_has_rows = m_tile * kTileM + quad * 32 < args.M;
+            RowState st;
+            st.m = -INFINITY; st.s = 0.f; st.t = 0.f; st.arg = 0x7fffffff;
+            for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
+                const int tu0 = u0 + tile * (kTileN / kUnit);
+                const int tun = min(kTileN / kUnit, u1 - tu0);
+                const uint32_t buf = tile_count & 1u;
+                const uint32_t acc_phase = (tile_count >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), acc_phase, ctl, args.status)) { alive = false; break; }
+                tc_fence_after_sync();
+                if (warp_has_rows) {
+                    const int v0 = tu0 * kUnit;
+                    for (int u = 0; u < tun; ++u) {
+                        uint32_t raw[16];
+                        tmem_ld16(lane_addr + buf * kTileN + u * kUnit, raw);
+                        tmem_ld_wait();
+                        const int col0 = v0 + u * kUnit;
+                        const int n = args.V - col0;
+                        if (n >= kUnit) fold16<true>(st, raw, col0, kUnit);
+                        else fold16<false>(st, raw, col0, n);
+                    }
+                }
+                tc_fence_before_sync();
+                mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
+            }
+            if (alive && row < args.M)
+                args.partials[(size_t)row * args.splits + q] = make_float4(st.m, st.s, st.t, __int_as_float(st.arg));
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------- merge kernel
+// One warp per row: combines the row's `splits` partial states (ascending vocabulary ranges) in
+// fp64 and writes token, confidence, entropy and planning-vocabulary membership.
+__global__ void __launch_bounds__(256)
+pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int splits,
+                       const uint32_t *__restrict__ plan_bitmap, int32_t *__restrict__ tok,
+                       float *__restrict__ conf, float *__restrict__ ent, uint8_t *__restrict__ in_plan)
+{
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= M) return;
+    const float4 *p = partials + (size_t)row * splits;
+    // lane-local pass: only the max and its lowest id
+    float m = -INFINITY;
+    int arg = 0x7fffffff;
+    for (int i = lane; i < splits; i += 32) {
+        const float4 v = p[i];
+        const int a = __float_as_int(v.w);
+        if (v.y > 0.f && (v.x > m || (v.x == m && a < arg))) { m = v.x; arg = a; }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
+        const int a2 = __shfl_xor_sync(0xffffffffu, arg, o);
+        if (m2 > m || (m2 == m && a2 < arg)) { m = m2; arg = a2; }
+    }
+    // rescale every partial to the global max and add
+    double s = 0.0, t = 0.0;
+    for (int i = lane; i < splits; i += 32) {
+        const float4 v = p[i];
+        if (v.y > 0.f) {
+            const double d = (double)v.x - (double)m;
+            const double c = exp(d);
+            s += (double)v.y * c;
+            t += ((double)v.z + d * (double)v.y) * c;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        s += __shfl_xor_sync(0xffffffffu, s, o);
+        t += __shfl_xor_sync(0xffffffffu, t, o);
+    }
+    if (lane == 0) {
+        tok[row] = arg;
+        conf[row] = (float)(1.0 / s);
+        if (ent) ent[row] = (float)(log(s) - t / s);
+        if (in_plan) in_plan[row] = (uint8_t)((plan_bitmap[arg >> 5] >> (arg & 31)) & 1u);
+    }
+}
+
+// ---------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// bf16 matrix [rows][cols] row-major, box = box_rows x 64 columns, 128-byte swizzle, zero fill outside.
+int make_tensor_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return PVF_ERR_CUDA;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
+    cuuint32_t elem[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PVF_OK : PVF_ERR_CUDA;
+}
+
+}  // namespace
+
+pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm)
+{
+    pvf_score_geometry g;
+    g.m_tiles = (M + kTileM - 1) / kTileM;
+    g.units = (V + kUnit - 1) / kUnit;
+    g.a_rows = g.m_tiles == 1 ? ((M + 7) / 8) * 8 : kTileM;
+    if (g.m_tiles == 0) { g.mb = g.splits = g.waves = g.ctas = 0; return g; }
+    // Pick the number of waves: cost = waves * max(per-block MMA work, HBM time of one W pass).
+    const double flops_per_sm = 1.0e13, hbm = 6.0e12;
+    double best_cost = 0.0;
+    int best_waves = 0, best_mb = 0, best_splits = 0;
+    for (int waves = 1; waves <= g.m_tiles; ++waves) {
+        const int mb = (g.m_tiles + waves - 1) / waves;
+        if (mb > n_sm || mb > kMaxConcurrentTiles) continue;
+        if ((g.m_tiles + mb - 1) / mb != waves) continue;          // same mb already seen with fewer waves
+        int splits = n_sm / mb;
+        if (splits > g.units) splits = g.units;
+        const int units_per_block = (g.units + splits - 1) / splits;
+        const double t_mma = (double)units_per_block * kUnit * kTileM * 2.0 * D / flops_per_sm;
+        const double t_hbm = 2.0 * V * (double)D / hbm;
+        const double cost = waves * (t_mma > t_hbm ? t_mma : t_hbm);
+        if (best_waves == 0 || cost < best_cost * 0.999) {
+            best_cost = cost; best_waves = waves; best_mb = mb; best_splits = splits;
+        }
+    }
+    g.waves = best_waves; g.mb = best_mb; g.splits = best_splits;
+    g.ctas = g.mb * g.splits;
+    return g;
+}
+
+size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm)
+{
+    size_t worst = 0;
+    const int max_tiles = (shape->max_rows + kTileM - 1) / kTileM;
+    for (int t = 1; t <= max_tiles; ++t) {
+        const int rows = t * kTileM < shape->max_rows ? t * kTileM : shape->max_rows;
+        const pvf_score_geometry g = pvf_score_geometry_for(rows, shape->vocab, shape->hidden, n_sm);
+        const size_t need = (size_t)rows * g.splits * sizeof(float4);
+        worst = need > worst ? need : worst;
+    }
+    return worst;
+}
+
+int pvf_score_init(pvf_ctx *ctx)
+{
+    int rc = make_tensor_map(&ctx->tm_w_full, ctx->w_head, (uint64_t)ctx->shape.vocab, (uint64_t)ctx->shape.hidden, kTileN);
+    if (rc != PVF_OK) return rc;
+    rc = make_tensor_map(&ctx->tm_w_unit, ctx->w_head, (uint64_t)ctx->shape.vocab, (uint64_t)ctx->shape.hidden, kUnit);
+    if (rc != PVF_OK) return rc;
+    if (cudaFuncSetAttribute(pvf_score_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        return PVF_ERR_CUDA;
+    return PVF_OK;
+}
+
+extern "C" {
+
+int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int32_t *waves, int32_t *launches)
+{
+    if (!ctx || M < 0 || M > ctx->shape.max_rows) return PVF_ERR_INVALID;
+    const pvf_score_geometry g = pvf_score_geometry_for(M, ctx->shape.vocab, ctx->shape.hidden, ctx->n_sm);
+    if (ctas) *ctas = g.ctas;
+    if (splits) *splits = g.splits;
+    if (waves) *waves = g.waves;
+    if (launches) *launches = M > 0 ? 2 : 0;
+    return PVF_OK;
+}
+
+int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
+              int32_t *tok, float *conf, float *ent, uint8_t *in_plan, void *stream)
+{
+    if (!ctx || M < 0 || M > ctx->shape.max_rows) return PVF_ERR_INVALID;
+    if (M == 0) return PVF_OK;
+    if (!hidden || !tok || !conf) return PVF_ERR_INVALID;
+    if (((uintptr_t)hidden & 15) != 0) return PVF_ERR_ALIGN;
+    const int V = ctx->shape.vocab, D = ctx->shape.hidden;
+    const pvf_score_geometry g = pvf_score_geometry_for(M, V, D, ctx->n_sm);
+    if ((size_t)M * g.splits * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
+
+    CUtensorMap tm_h;
+    int rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)g.a_rows);
+    if (rc != PVF_OK) return rc;
+
+    ScoreArgs a;
+    a.M = M; a.V = V; a.D = D;
+    a.num_kb = (D + kBlockK - 1) / kBlockK;
+    a.units = g.units;
+    a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
+    a.a_rows = g.a_rows;
+    a.partials = ctx->partials;
+    a.status = &ctx->words->status;
+    cudaStream_t s = (cudaStream_t)stream;
+    pvf_score_gemm_kernel<<<g.ctas, kThreads, kSmemBytes, s>>>(tm_h, ctx->tm_w_full, ctx->tm_w_unit, a);
+    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
+    const int warps_per_block = 8;
+    pvf_score_merge_kernel<<<(M + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(
+        ctx->partials, M, g.splits, ctx->plan_bitmap, tok, conf, ent, in_plan);
+    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
+    return PVF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,213 @@
+"""The whole step (score -> commit -> select -> verification-pass score -> verify) on the synthetic
+configurations, GPU against oracle.  LLaDA-shaped cases score every row on the GPU in the launch
+geometry the benchmark times and check a sample of rows against the oracle one by one."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import score as oscore
+from oracle import step as ostep
+from paper_2601_12247_b200 import binding, synth
+from gpu_util import (FRAGILE, NEAR_TIE, check_score, check_score_properties, dev, make_ctx, params_of, t_i32, t_u8,
+                      to_np, upload_bits)
+
+pytestmark = pytest.mark.gpu
+
+
+def fragile_rows(conf, thresholds):
+    bad = np.zeros(len(conf), bool)
+    for t in thresholds:
+        bad |= np.abs(conf - float(np.float32(t))) < FRAGILE
+    return bad
+
+
+def full_step(ctx, st, flags=0):
+    """GPU step and oracle step, each on its own scores; decisions must agree on every sequence
+    that holds no near-tie or threshold-fragile row."""
+    p = st.params
+    prm = params_of(st, flags)
+    seg, pos, act = t_i32(st.seg_off), t_i32(st.row_pos), t_u8(st.active)
+    sc = ctx.score(upload_bits(st.h_bits))
+    cm = ctx.commit(prm, seg, pos, act, sc["tok"], sc["conf"])
+    sel = ctx.select_drafts(prm, seg, pos, act, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
+    torch.cuda.synchronize()
+
+    osc = oscore.score(st.w_bits, st.h_bits, st.plan_ids)
+    check_score(to_np(sc), osc, st.vocab, st.plan_ids)
+    force = bool(flags & binding.PVF_FORCE_PROGRESS)
+    ocm = ostep.commit(osc["conf"], osc["tok"], st.seg_off, st.row_pos, st.active, p["tau_high"], force)
+    osel = ostep.select_drafts(osc["conf"], osc["tok"], osc["in_plan"], ocm["commit"], st.seg_off, st.row_pos,
+                               st.active, p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], p["budget"])
+    bad_row = (osc["gap"] < NEAR_TIE) | fragile_rows(osc["conf"], [p["tau_high"], p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"]])
+    seq_ok = np.array([not bad_row[st.seg_off[b]:st.seg_off[b + 1]].any() for b in range(st.n_seq)])
+    # top-k fragility: K-th and (K+1)-th candidate closer than FRAGILE
+    for b in range(st.n_seq):
+        rows = np.arange(st.seg_off[b], st.seg_off[b + 1])
+        cand = [m for m in rows if st.active[m] and not ocm["commit"][m] and osc["in_plan"][m]
+                and np.float32(p["tau_plan_lo"]) <= osc["conf"][m] < np.float32(p["tau_plan_hi"])]
+        cs = sorted((osc["conf"][m] for m in cand), reverse=True)
+        K = p["budget"]
+        if len(cs) > K and cs[K - 1] - cs[K] < FRAGILE:
+            seq_ok[b] = False
+    g_cm, g_sel = to_np(cm), to_np(sel)
+    row_ok = np.repeat(seq_ok, np.diff(st.seg_off))
+    assert np.array_equal(g_cm["commit"][row_ok], ocm["commit"][row_ok])
+    for b in np.nonzero(seq_ok)[0]:
+        assert np.array_equal(g_sel["draft_rows"][b], osel["draft_rows"][b])
+        assert g_sel["route"][b] == osel["route"][b] and g_sel["n_drafts"][b] == osel["n_drafts"][b]
+    return sc, cm, sel, osc, ocm, osel, seq_ok
+
+
+def verify_pass(ctx, st, sc, cm, sel, osc, ocm, osel, seq_ok, flags=0):
+    p = st.params
+    prm = params_of(st, flags)
+    if not seq_ok.all():            # decisions differ legitimately somewhere: the layouts would not line up
+        pytest.skip("fragile sequence present")
+    v = synth.make_verify_pass(st, osel["rem_rows"], osel["rem_off"], osel["n_drafts"])
+    assert np.array_equal(v.v_off, osel["v_off"])
+    scv = ctx.score(upload_bits(v.hv_bits))
+    seg, pos = t_i32(st.seg_off), t_i32(st.row_pos)
+    ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"])
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    oscv = oscore.score(st.w_bits, v.hv_bits, st.plan_ids)
+    check_score(to_np(scv), oscv, st.vocab, st.plan_ids)
+    over = ostep.verify(osc["tok"], ocm["commit"], st.seg_off, st.row_pos, osel["rem_rows"], osel["rem_off"],
+                        osel["v_off"], osel["draft_rows"], osel["n_drafts"], osel["route"], oscv["tok"], oscv["conf"],
+                        p["tau_high"], p["budget"])
+    gv = to_np(ver)
+    bad_v = (oscv["gap"] < NEAR_TIE) | fragile_rows(oscv["conf"], [p["tau_high"]])
+    margins = ostep.c_total_margins(osel["rem_rows"], osel["rem_off"], osel["v_off"], osel["draft_rows"],
+                                    osel["n_drafts"], osel["route"], oscv["conf"], over["accept"])
+    n_checked = 0
+    for b in range(st.n_seq):
+        if bad_v[osel["v_off"][b]:osel["v_off"][b + 1]].any() or margins[b] < 1e-3:
+            continue
+        n_checked += 1
+        assert np.array_equal(gv["accept"][b], over["accept"][b]) and gv["choice"][b] == over["choice"][b]
+        rows = slice(st.seg_off[b], st.seg_off[b + 1])
+        assert np.array_equal(gv["final_commit"][rows], over["final_commit"][rows])
+    assert n_checked >= (st.n_seq + 1) // 2
+    return over
+
+
+@pytest.mark.parametrize("stress", [False, True])
+def test_config0_full_step(stress):
+    st = synth.config0(stress=stress)
+    ctx = make_ctx(st.w_bits, st.plan_ids, 4096)
+    parts = full_step(ctx, st)
+    verify_pass(ctx, st, *parts)
+    ctx.close()
+
+
+@pytest.mark.parametrize("stress", [False, True])
+def test_config2_and_3_at_small_vocab(stress):
+    # the batched and large-batch row layouts at a vocabulary the oracle scores in seconds
+    w = synth.make_w(2002, 8192, 256)
+    ctx = make_ctx(w, synth.make_plan_ids(1002, 8192, 2048), 8192, 64, 16)
+    st2 = synth.config2(stress=stress, w_bits=w, vocab=8192, hidden=256)
+    over = verify_pass(ctx, st2, *full_step(ctx, st2))
+    ctx.close()
+    st3 = synth.config3(stress=stress, w_bits=w, vocab=8192, hidden=256, n_seq=8, gen_len=128)
+    ctx = make_ctx(w, st3.plan_ids, 8192, 64, 16)
+    verify_pass(ctx, st3, *full_step(ctx, st3))
+    ctx.close()
+
+
+# ------------------------------------------------------------------------------ LLaDA shape
+@pytest.fixture(scope="module")
+def llada():
+    w_bits = synth.make_w(1001, synth.LLADA_VOCAB, synth.LLADA_HIDDEN)
+    plan = synth.make_plan_ids(1001, synth.LLADA_VOCAB, 2048)
+    ctx = make_ctx(w_bits, plan, 32768, 64, 16)
+    yield w_bits, plan, ctx
+    ctx.close()
+
+
+def sampled_parity(ctx, st, w_bits, plan, sample):
+    h = upload_bits(st.h_bits)
+    got = to_np(ctx.score(h))
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    check_score_properties(got, st.vocab, plan)
+    want = oscore.score(w_bits, st.h_bits[sample], plan)
+    check_score(got, want, st.vocab, plan, rows=sample)
+    return got
+
+
+def test_config1a_every_row(llada):
+    w_bits, plan, ctx = llada
+    st = synth.config1("a", w_bits=w_bits)
+    assert ctx.score_plan(32)["ctas"] == torch.cuda.get_device_properties(0).multi_processor_count
+    parts = full_step(ctx, st)
+    assert parts[-1].all()
+
+
+def test_config1a_stress_every_row(llada):
+    w_bits, plan, ctx = llada
+    st = synth.config1("a", stress=True, w_bits=w_bits)
+    full_step(ctx, st)
+
+
+def test_config1b_sampled(llada):
+    w_bits, plan, ctx = llada
+    st = synth.config1("b", w_bits=w_bits)
+    sampled_parity(ctx, st, w_bits, plan, np.array([0, 31, 32, 127, 128, 129, 200, 255]))
+
+
+def test_config2_sampled_rows_and_decisions_on_gpu_scores(llada):
+    w_bits, plan, ctx = llada
+    st = synth.config2(w_bits=w_bits)
+    M = st.n_rows
+    got = sampled_parity(ctx, st, w_bits, plan, np.unique(np.linspace(0, M - 1, 12).astype(int)))
+    # decisions are integer work: on the GPU's own fp32 scores they must equal the oracle's exactly
+    p = st.params
+    prm = params_of(st)
+    seg, pos, act = t_i32(st.seg_off), t_i32(st.row_pos), t_u8(st.active)
+    sc = ctx.score(upload_bits(st.h_bits))
+    cm = ctx.commit(prm, seg, pos, act, sc["tok"], sc["conf"])
+    sel = ctx.select_drafts(prm, seg, pos, act, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
+    ocm = ostep.commit(got["conf"], got["tok"], st.seg_off, st.row_pos, st.active, p["tau_high"])
+    osel = ostep.select_drafts(got["conf"], got["tok"], got["in_plan"], ocm["commit"], st.seg_off, st.row_pos,
+                               st.active, p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], p["budget"])
+    assert np.array_equal(to_np(cm)["commit"], ocm["commit"])
+    gs = to_np(sel)
+    for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+        assert np.array_equal(gs[k], osel[k]), k
+    v = synth.make_verify_pass(st, osel["rem_rows"], osel["rem_off"], osel["n_drafts"])
+    scv = ctx.score(upload_bits(v.hv_bits))
+    ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"])
+    gscv = to_np(scv)
+    over = ostep.verify(got["tok"], ocm["commit"], st.seg_off, st.row_pos, osel["rem_rows"], osel["rem_off"],
+                        osel["v_off"], osel["draft_rows"], osel["n_drafts"], osel["route"], gscv["tok"], gscv["conf"],
+                        p["tau_high"], p["budget"])
+    gv = to_np(ver)
+    for k in ("accept", "choice", "final_commit"):
+        assert np.array_equal(gv[k], over[k]), k
+    Mv = v.hv_bits.shape[0]
+    if Mv:
+        rows = np.unique(np.linspace(0, Mv - 1, 6).astype(int))
+        check_score(gscv, oscore.score(w_bits, v.hv_bits[rows], plan), st.vocab, plan, rows=rows)
+
+
+def test_config3_large_batch_sampled(llada):
+    w_bits, plan, ctx = llada
+    st = synth.config3(w_bits=w_bits)
+    assert st.n_rows == 32768
+    geo = ctx.score_plan(st.n_rows)
+    assert geo["waves"] >= 2 and geo["ctas"] <= torch.cuda.get_device_properties(0).multi_processor_count
+    sample = np.array([0, 127, 128, 4735, 4736, 16383, 20000, 32767])
+    got = sampled_parity(ctx, st, w_bits, plan, sample)
+    p = st.params
+    prm = params_of(st)
+    seg, pos, act = t_i32(st.seg_off), t_i32(st.row_pos), t_u8(st.active)
+    sc = dict(tok=t_i32(got["tok"]), conf=torch.from_numpy(got["conf"]).to(dev()), in_plan=t_u8(got["in_plan"]))
+    cm = ctx.commit(prm, seg, pos, act, sc["tok"], sc["conf"])
+    sel = ctx.select_drafts(prm, seg, pos, act, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
+    ocm = ostep.commit(got["conf"], got["tok"], st.seg_off, st.row_pos, st.active, p["tau_high"])
+    osel = ostep.select_drafts(got["conf"], got["tok"], got["in_plan"], ocm["commit"], st.seg_off, st.row_pos,
+                               st.active, p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], p["budget"])
+    assert np.array_equal(to_np(cm)["commit"], ocm["commit"])
+    gs = to_np(sel)
+    for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+        assert np.array_equal(gs[k], osel[k]), k

@@ -1,0 +1,94 @@
+"""pvf_score against the fp64 oracle, element by element, through the C interface."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import score as oscore
+from paper_2601_12247_b200 import binding, synth
+from gpu_util import check_score, check_score_properties, dev, make_ctx, to_np, upload_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def run_and_compare(w_bits, h_bits, plan_ids, max_rows=None, rows=None):
+    ctx = make_ctx(w_bits, plan_ids, max_rows or max(1, h_bits.shape[0]))
+    h = upload_bits(h_bits)
+    got = to_np(ctx.score(h))
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    again = to_np(ctx.score(h))
+    torch.cuda.synchronize()
+    for k in got:
+        assert np.array_equal(got[k], again[k]), "run-to-run difference in " + k
+    sub = h_bits if rows is None else h_bits[rows]
+    want = oscore.score(w_bits, sub, plan_ids)
+    near = check_score(got, want, w_bits.shape[0], plan_ids, rows)
+    check_score_properties(got, w_bits.shape[0], plan_ids)
+    ctx.close()
+    return got, want, near
+
+
+@pytest.mark.parametrize("stress", [False, True])
+def test_config0_tiny(stress):
+    st = synth.config0(stress=stress)
+    got, want, near = run_and_compare(st.w_bits, st.h_bits, st.plan_ids)
+    assert near <= 2
+
+
+@pytest.mark.parametrize("V,D,M", [(4096, 256, 1), (4096, 256, 7), (4096, 256, 128), (4096, 256, 129),
+                                   (5000, 200, 150), (1000, 64, 33), (16, 8, 3), (70000, 512, 300)])
+def test_ragged_shapes(V, D, M):
+    # several row tiles, vocabulary not a multiple of 16, hidden size not a multiple of 64
+    pos = np.arange(M)
+    st = synth.build_step("ragged", 4242, V, D, min(64, V), [(pos, np.ones(M, np.uint8))], M, M,
+                          dict(tau_high=0.9, budget=4), amp_max=40.0 * (256.0 / D) ** 0.5)
+    run_and_compare(st.w_bits, st.h_bits, st.plan_ids)
+
+
+def test_uniform_and_peaked_closed_forms():
+    # all-zero hidden state -> p = 1/V, H = ln V, token 0;  W = c*I -> one logit a*c, the rest 0
+    V = 256
+    w = synth.f32_to_bf16_bits(0.5 * np.eye(V, dtype=np.float32))
+    h = np.zeros((3, V), np.float32); h[1, 17] = 8.0; h[2, 255] = 30.0
+    ctx = make_ctx(w, [17], 8)
+    got = to_np(ctx.score(upload_bits(synth.f32_to_bf16_bits(h))))
+    assert got["tok"].tolist() == [0, 17, 255] and got["in_plan"].tolist() == [0, 1, 0]
+    Z = np.exp(4.0) + V - 1
+    assert abs(got["conf"][0] - 1.0 / V) < 1e-6 and abs(got["ent"][0] - np.log(V)) < 1e-4
+    assert abs(got["conf"][1] - np.exp(4.0) / Z) < 1e-5 and abs(got["ent"][1] - (np.log(Z) - 4.0 * np.exp(4.0) / Z)) < 1e-4
+    Z2 = np.exp(15.0) + V - 1
+    assert abs(got["conf"][2] - np.exp(15.0) / Z2) < 1e-5
+    assert abs(got["ent"][2] - (np.log(Z2) - 15.0 * np.exp(15.0) / Z2)) < 1e-4
+    ctx.close()
+
+
+def test_exact_tie_goes_to_lowest_id_across_ranges():
+    # identical weight rows far apart in the vocabulary: equal logits in different blocks' ranges
+    V, D = 4096, 64
+    w = synth.make_w(9, V, D)
+    w[3000] = w[10]; w[4095] = w[10]
+    h = (synth.bf16_bits_to_f32(w[10]).astype(np.float32) * 400.0)[None, :]
+    ctx = make_ctx(w, [10], 8)
+    got = to_np(ctx.score(upload_bits(synth.f32_to_bf16_bits(h))))
+    assert got["tok"][0] == 10 and got["in_plan"][0] == 1
+    ctx.close()
+
+
+def test_argument_errors_launch_nothing():
+    st = synth.config0()
+    ctx = make_ctx(st.w_bits, st.plan_ids, 64)
+    h = upload_bits(st.h_bits)
+    out = ctx.score(h[:0])                                        # M = 0 is a no-op
+    assert out["tok"].numel() == 0
+    big = upload_bits(np.concatenate([st.h_bits, st.h_bits]))
+    with pytest.raises(binding.PvfError) as e:
+        ctx.score(big)                                            # above max_rows
+    assert e.value.code == binding.PVF_ERR_INVALID
+    flat = torch.empty(64 * 256 + 8, dtype=torch.bfloat16, device=dev())
+    mis = flat[1:1 + 64 * 256].view(64, 256)                      # 2-byte offset: not 16-byte aligned
+    with pytest.raises(binding.PvfError) as e:
+        ctx.score(mis)
+    assert e.value.code == binding.PVF_ERR_ALIGN
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    ctx.close()
