@@ -1,0 +1,381 @@
+#!/usr/bin/env python
+"""Benchmark of the fused PVF step on one node.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1a|cfg1b|cfg2|cfg3]
+
+A step is one pass of the whole hot path over one synthetic batch, through the C interface:
+    pvf_score(H) -> pvf_commit -> pvf_select_drafts -> pvf_score(Hv, verification pass) -> pvf_verify
+Default workload (cfg1a): LLaDA-8B-shaped single step -- vocabulary 126464, hidden 4096, bf16, one
+sequence, the 32 masked positions of the active block, budget 4.  The metric is masked positions
+scored per second per fused step (draft-pass rows / step time); the verification-pass rows are
+reported beside it.  Inputs are seeded synthetic tensors; W (1.04 GB) is far larger than L2, so
+every step streams it from HBM again.
+
+With N > 1 (torchrun) every rank runs the same step on its own batch (independent replicas, no
+collective on the data path); the value is the sum over ranks divided by the slowest rank's time.
+
+`--impl reference` times the CPU fp64 oracle (oracle/) on the same workload's rows.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "masked positions scored/s per fused PVF step"
+UNIT = "positions/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def make_workload(name: str, synth, seed_w: int = 1001):
+    w_bits = synth.make_w(seed_w, synth.LLADA_VOCAB, synth.LLADA_HIDDEN)
+    if name == "cfg1a":
+        st = synth.config1("a", w_bits=w_bits)
+    elif name == "cfg1b":
+        st = synth.config1("b", w_bits=w_bits)
+    elif name == "cfg2":
+        st = synth.config2(w_bits=w_bits)
+    elif name == "cfg3":
+        st = synth.config3(w_bits=w_bits)
+    else:
+        raise SystemExit("unknown workload " + name)
+    return st
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str, period_ms: int = 100):
+        self.cmd = ["nvidia-smi", "-i", gpu_id, "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                    "-lms", str(period_ms)]
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(self.cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                    samples=len(sm), power_w_max=float(max(power)))
+
+
+# ------------------------------------------------------------------------------------ reference arm
+def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from oracle import score as oscore
+    from oracle import step as ostep
+    from paper_2601_12247_b200 import synth
+    st = make_workload(args.workload, synth)
+    p = st.params
+    cores = oscore.threads()
+    # per-step sample: the first `rows` rows of the workload, sized from one probe row so that the
+    # whole run stays within a few minutes
+    t0 = time.perf_counter()
+    oscore.score(st.w_bits, st.h_bits[:1], st.plan_ids)
+    per_row = time.perf_counter() - t0
+    budget_s = 150.0
+    rows = int(max(1, min(st.n_rows, budget_s / max(per_row, 1e-6) / max(1, args.steps + args.warmup))))
+
+    def one_step():
+        sc = oscore.score(st.w_bits, st.h_bits[:rows], st.plan_ids)
+        n_seq_rows = rows
+        seg = np.array([0, n_seq_rows], np.int32)
+        cm = ostep.commit(sc["conf"], sc["tok"], seg, st.row_pos[:rows], st.active[:rows], p["tau_high"])
+        ostep.select_drafts(sc["conf"], sc["tok"], sc["in_plan"], cm["commit"], seg, st.row_pos[:rows],
+                            st.active[:rows], p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], p["budget"])
+
+    for _ in range(args.warmup):
+        one_step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_step()
+    dt = time.perf_counter() - t0
+    value = rows * args.steps / dt
+    sample = "first %d of %d draft-pass rows per step: fp64 score + commit + draft selection" % (rows, st.n_rows)
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * dt / args.steps, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=args.workload, vocab=st.vocab, hidden=st.hidden, rows_per_step=rows),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------ our arm
+def run_ours(args):
+    import torch
+    from paper_2601_12247_b200 import binding, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=dev)
+    peaks = load_peaks()
+
+    st = make_workload(args.workload, synth)
+    p = st.params
+    M, V, D = st.n_rows, st.vocab, st.hidden
+    K = int(p["budget"])
+    max_rows = 8192 if M <= 4096 else M * (2 + K)       # room for the verification pass
+    ctx = binding.Context(binding.bf16_from_bits(st.w_bits, dev), st.plan_ids, max_rows, max(64, st.n_seq), max(16, K))
+    prm = binding.make_params(p["tau_high"], p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], K)
+    i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
+    seg, pos = i32(st.seg_off), i32(st.row_pos)
+    act = torch.from_numpy(np.ascontiguousarray(st.active)).to(dev)
+    h_host = binding.bf16_from_bits(st.h_bits, "cpu").pin_memory()
+    h = h_host.to(dev)
+
+    # One untimed draft pass fixes the verification-pass layout (R_b and K_t of every sequence).
+    sc = ctx.score(h)
+    cm = ctx.commit(prm, seg, pos, act, sc["tok"], sc["conf"])
+    sel = ctx.select_drafts(prm, seg, pos, act, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
+    torch.cuda.synchronize()
+    sel_np = {k: v.cpu().numpy() for k, v in sel.items()}
+    n_rem = int(sel_np["rem_off"][-1])
+    vp = synth.make_verify_pass(st, sel_np["rem_rows"][:n_rem], sel_np["rem_off"], sel_np["n_drafts"])
+    Mv = int(vp.hv_bits.shape[0])
+    hv_host = binding.bf16_from_bits(vp.hv_bits, "cpu").pin_memory() if Mv else None
+    hv = hv_host.to(dev) if Mv else None
+    if Mv > ctx.shape.max_rows:
+        raise SystemExit("verification pass larger than the context")
+
+    # preallocated outputs: the timed loop allocates nothing
+    def outs(n):
+        return dict(tok=torch.empty(n, dtype=torch.int32, device=dev), conf=torch.empty(n, dtype=torch.float32, device=dev),
+                    ent=torch.empty(n, dtype=torch.float32, device=dev), in_plan=torch.empty(n, dtype=torch.uint8, device=dev))
+    o_sc, o_scv = outs(M), outs(max(Mv, 1))
+    o_cm = dict(commit=torch.empty(M, dtype=torch.uint8, device=dev), n_commit=torch.empty(st.n_seq, dtype=torch.int32, device=dev))
+    o_sel = {k: torch.empty_like(v) for k, v in sel.items()}
+    o_ver = dict(accept=torch.empty((st.n_seq, K), dtype=torch.uint8, device=dev),
+                 choice=torch.empty(st.n_seq, dtype=torch.int32, device=dev),
+                 final_commit=torch.empty(M, dtype=torch.uint8, device=dev))
+    ev_pairs = []
+    ev_pool = []
+    for _ in range(2 * args.steps):                # created (and first recorded) outside the timed region
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); b.record()
+        ev_pool.append((a, b))
+    torch.cuda.synchronize()
+
+    def step(h_dev, hv_dev, timed_events=False):
+        launches = 0
+        if timed_events:
+            a, b = ev_pool.pop()
+            ctx.set_score_events(a, b); ev_pairs.append((a, b, M))
+        ctx.score(h_dev, o_sc); launches += 2
+        ctx.commit(prm, seg, pos, act, o_sc["tok"], o_sc["conf"], out=o_cm); launches += 1
+        ctx.select_drafts(prm, seg, pos, act, o_sc["tok"], o_sc["conf"], o_sc["in_plan"], o_cm["commit"], out=o_sel); launches += 1
+        if Mv:
+            if timed_events:
+                a, b = ev_pool.pop()
+                ctx.set_score_events(a, b); ev_pairs.append((a, b, Mv))
+            ctx.score(hv_dev, o_scv); launches += 2
+        ctx.verify(prm, seg, pos, o_sel, o_sc["tok"], o_scv["tok"], o_scv["conf"], o_cm["commit"], out=o_ver); launches += 1
+        return launches
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- device-resident timing
+    for _ in range(max(args.warmup, 3)):
+        step(h, hv)
+    barrier()
+    props = torch.cuda.get_device_properties(dev)
+    if hasattr(props, "uuid"):
+        gpu_id = "GPU-" + str(props.uuid)
+    else:
+        visible = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+        gpu_id = visible.split(",")[local_rank] if visible else str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches = 0
+    e0.record()
+    for _ in range(args.steps):
+        launches += step(h, hv, timed_events=True)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ctx.set_score_events(None, None)
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    status = ctx.last_status()
+    value = world * M * args.steps / (ms * 1e-3)
+
+    # roofline of the dominant kernel (the score GEMM), from the events recorded in the timed region
+    gemm_ms = sum(a.elapsed_time(b) for a, b, _ in ev_pairs)
+    rows_scored = sum(r for _, _, r in ev_pairs)
+    n_gemm = len(ev_pairs)
+    alg_bytes = sum(2.0 * V * D + 2.0 * r * D + 13.0 * r + V / 8.0 for _, _, r in ev_pairs)
+    alg_flops = sum(2.0 * r * V * D for _, _, r in ev_pairs)
+    t_gemm = gemm_ms * 1e-3
+    hbm_time = alg_bytes / (peaks["hbm_gbs"] * 1e9)
+    tc_time = alg_flops / (peaks["bf16_tflops_sustained"] * 1e12)
+    if hbm_time >= tc_time:
+        roof = dict(bound="hbm", achieved=alg_bytes / t_gemm / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+    else:
+        roof = dict(bound="tensor", achieved=alg_flops / t_gemm / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof.update(traffic=None, kernel="pvf_score_gemm_kernel", launches=n_gemm, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
+                algorithmic_bytes_per_launch=alg_bytes / max(n_gemm, 1), peak_source=peaks["source"] +
+                (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy bandwidth)"))
+
+    # ---------------- end to end: inputs start in pinned host memory, results end in host memory
+    n_e2e = max(3, min(args.steps, 200))
+    host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in
+                dict(tok=o_sc["tok"], conf=o_sc["conf"], commit=o_cm["commit"], draft_rows=o_sel["draft_rows"],
+                     n_drafts=o_sel["n_drafts"], route=o_sel["route"], v_off=o_sel["v_off"], accept=o_ver["accept"],
+                     choice=o_ver["choice"], final_commit=o_ver["final_commit"]).items()}
+    h_dev2 = torch.empty_like(h)
+    hv_dev2 = torch.empty_like(hv) if Mv else None
+
+    def e2e_step():
+        h_dev2.copy_(h_host, non_blocking=True)
+        if Mv:
+            hv_dev2.copy_(hv_host, non_blocking=True)
+        step(h_dev2, hv_dev2)
+        for k, src in (("tok", o_sc["tok"]), ("conf", o_sc["conf"]), ("commit", o_cm["commit"]),
+                       ("draft_rows", o_sel["draft_rows"]), ("n_drafts", o_sel["n_drafts"]), ("route", o_sel["route"]),
+                       ("v_off", o_sel["v_off"]), ("accept", o_ver["accept"]), ("choice", o_ver["choice"]),
+                       ("final_commit", o_ver["final_commit"])):
+            host_out[k].copy_(src, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(n_e2e):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    h2d = int(h_host.numel() * 2 + (hv_host.numel() * 2 if Mv else 0))
+    d2h = int(sum(v.numel() * v.element_size() for v in host_out.values()))
+    e2e = dict(value=world * M * n_e2e / (ms_e2e * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+               steps=n_e2e, ms_per_step=ms_e2e / n_e2e)
+
+    # ---------------- CPU baseline: the oracle on the same step (rank 0, single-GPU runs only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        from oracle import score as oscore
+        from oracle import step as ostep
+        rows = min(M, args.cpu_rows)
+        rows_v = min(Mv, args.cpu_rows)
+        t0 = time.perf_counter()
+        osc = oscore.score(st.w_bits, st.h_bits[:rows], st.plan_ids)
+        if rows == M:
+            ocm = ostep.commit(osc["conf"], osc["tok"], st.seg_off, st.row_pos, st.active, p["tau_high"])
+            ostep.select_drafts(osc["conf"], osc["tok"], osc["in_plan"], ocm["commit"], st.seg_off, st.row_pos,
+                                st.active, p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], K)
+        if rows_v:
+            oscore.score(st.w_bits, vp.hv_bits[:rows_v], st.plan_ids)
+        dt = time.perf_counter() - t0
+        frac = (rows + rows_v) / float(M + Mv)
+        cpu = dict(value=M * frac / dt, unit=UNIT, cores=oscore.threads(), kind="oracle", seconds=dt,
+                   sample="%d of %d draft-pass rows and %d of %d verification-pass rows of the same step, fp64 score%s"
+                          % (rows, M, rows_v, Mv, " + commit + draft selection" if rows == M else ""))
+
+    if rank == 0:
+        geo = ctx.score_plan(M)
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                    ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                    data="synthetic",
+                    config=dict(workload=args.workload + " (" + st.name + ")", vocab=V, hidden=D, n_seq=st.n_seq,
+                                draft_rows=M, verify_rows=Mv, budget=K, tau_high=p["tau_high"],
+                                step="score+commit+select+score(verify)+verify",
+                                l2="inputs larger than L2: the 1.04 GB weight matrix is streamed from HBM every score call",
+                                parallelism="replicas" if world > 1 else "single GPU", score_geometry=geo),
+                    clocks=dict(sm_mhz=clocks.get("sm_mhz"), sm_max_mhz=clocks.get("sm_max_mhz"),
+                                reasons=clocks.get("reasons", []), samples=clocks.get("samples", 0),
+                                power_w_max=clocks.get("power_w_max")),
+                    e2e=e2e, gpu_launches=launches, roofline=roof, cpu_baseline=cpu, status=status)
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg3"])
+    ap.add_argument("--cpu-rows", type=int, default=256, help="rows per pass the CPU baseline scores")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -111,6 +111,14 @@ int pvf_last_status(pvf_ctx *ctx, int32_t *status);
 int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int32_t *waves, int32_t *launches);
 
 /*
+ * Timing hook for benchmarks.  While both events (cudaEvent_t passed as void*) are non-NULL, every
+ * pvf_score call records `start` immediately before and `stop` immediately after its GEMM kernel on
+ * the call's stream, so the kernel can be timed alone inside a longer step.  NULL, NULL switches it
+ * off (the default).  The events stay owned by the caller.
+ */
+int pvf_set_score_events(pvf_ctx *ctx, void *start, void *stop);
+
+/*
  * pvf_score -- the vocabulary pass of one forward (Section 2 "confidence-based parallel decoding";
  * Section 3, definitions of y^_t^i, p_t^i and H_i; Section 4.1, "y^ in P^plan").
  *
@@ -173,7 +181,8 @@ int pvf_select_drafts(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t
  * AR route: accept[b][k-1] = for all r <= k: tok_v[k][row of fill r] == tok[fill r];
  *   choice[b] = largest accepted k, 0 if none.
  * final_commit = commit, plus draft `choice` (planning) or fills 1..choice (AR).  y as in pvf_commit,
- * written at every final_commit row.  accept entries beyond n_drafts[b] are 0.
+ * written at every final_commit row.  accept entries beyond n_drafts[b] are 0.  tok_v, conf_v and
+ * rem_rows are only read for sequences that have drafts (they may be NULL when v_off[n_seq] = 0).
  */
 int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
                const int32_t *seg_off, const int32_t *row_pos,

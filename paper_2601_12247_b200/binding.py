@@ -58,6 +58,7 @@ def load() -> ctypes.CDLL:
         lib.pvf_create.argtypes = [ctypes.POINTER(vp), ps, vp, vp, i32, vp, sz]; lib.pvf_create.restype = ctypes.c_int
         lib.pvf_destroy.argtypes = [vp]; lib.pvf_destroy.restype = ctypes.c_int
         lib.pvf_last_status.argtypes = [vp, ctypes.POINTER(i32)]; lib.pvf_last_status.restype = ctypes.c_int
+        lib.pvf_set_score_events.argtypes = [vp, vp, vp]; lib.pvf_set_score_events.restype = ctypes.c_int
         lib.pvf_score_plan.argtypes = [vp, i32] + [ctypes.POINTER(i32)] * 4; lib.pvf_score_plan.restype = ctypes.c_int
         lib.pvf_score.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]; lib.pvf_score.restype = ctypes.c_int
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
@@ -133,6 +134,15 @@ class Context:
         st = ctypes.c_int32()
         _check(self.lib.pvf_last_status(self.handle, ctypes.byref(st)), "pvf_last_status")
         return int(st.value)
+
+    def set_score_events(self, start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]):
+        """Timing hook: events recorded around the GEMM kernel of every following score call."""
+        for ev in (start, stop):
+            if ev is not None and not ev.cuda_event:
+                ev.record()                      # torch creates the CUDA event lazily, on first record
+        a = None if start is None else ctypes.c_void_p(start.cuda_event)
+        b = None if stop is None else ctypes.c_void_p(stop.cuda_event)
+        _check(self.lib.pvf_set_score_events(self.handle, a, b), "pvf_set_score_events")
 
     def score_plan(self, M: int) -> Dict[str, int]:
         v = [ctypes.c_int32() for _ in range(4)]

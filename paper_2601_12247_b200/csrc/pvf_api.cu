@@ -103,6 +103,8 @@ int pvf_create(pvf_ctx **out, const pvf_shape *shape, const void *w_head,
     ctx->plan_bitmap = (uint32_t *)(ctx->workspace + l.bitmap_off);
     ctx->partials = (float4 *)(ctx->workspace + l.partials_off);
     ctx->partials_bytes = l.partials_bytes;
+    ctx->ev_start = nullptr;
+    ctx->ev_stop = nullptr;
 
     std::vector<uint32_t> bitmap(l.bitmap_bytes / 4, 0u);
     for (int32_t i = 0; i < n_plan; ++i) bitmap[plan_ids_host[i] >> 5] |= 1u << (plan_ids_host[i] & 31);

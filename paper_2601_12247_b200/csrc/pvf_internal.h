@@ -30,6 +30,7 @@ struct pvf_ctx {
     size_t partials_bytes;
     CUtensorMap tm_w_full;  // W as [V][D], box 256 rows x 64 columns, 128-byte swizzle
     CUtensorMap tm_w_unit;  // same tensor, box 16 rows x 64 columns
+    cudaEvent_t ev_start, ev_stop;   // optional timing hook around the GEMM kernel
 };
 
 // Work split of pvf_score for M rows on n_sm SMs (see pvf_score.cu).

@@ -554,6 +554,14 @@ int pvf_score_init(pvf_ctx *ctx)
 
 extern "C" {
 
+int pvf_set_score_events(pvf_ctx *ctx, void *start, void *stop)
+{
+    if (!ctx || ((start == nullptr) != (stop == nullptr))) return PVF_ERR_INVALID;
+    ctx->ev_start = (cudaEvent_t)start;
+    ctx->ev_stop = (cudaEvent_t)stop;
+    return PVF_OK;
+}
+
 int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int32_t *waves, int32_t *launches)
 {
     if (!ctx || M < 0 || M > ctx->shape.max_rows) return PVF_ERR_INVALID;
@@ -589,8 +597,11 @@ int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
     a.partials = ctx->partials;
     a.status = &ctx->words->status;
     cudaStream_t s = (cudaStream_t)stream;
+    const bool timed = ctx->ev_start && ctx->ev_stop;
+    if (timed && cudaEventRecord(ctx->ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
     pvf_score_gemm_kernel<<<g.ctas, kThreads, kSmemBytes, s>>>(tm_h, ctx->tm_w_full, ctx->tm_w_unit, a);
     if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
+    if (timed && cudaEventRecord(ctx->ev_stop, s) != cudaSuccess) return PVF_ERR_CUDA;
     const int warps_per_block = 8;
     pvf_score_merge_kernel<<<(M + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(
         ctx->partials, M, g.splits, ctx->plan_bitmap, tok, conf, ent, in_plan);

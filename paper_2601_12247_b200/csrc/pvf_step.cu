@@ -390,7 +390,7 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
     if (n_seq == 0) return M == 0 ? PVF_OK : PVF_ERR_INVALID;
     if (!seg_off || !rem_off || !v_off || !n_drafts || !route || !commit || !choice || !final_commit ||
         (params->budget > 0 && (!draft_rows || !accept)) ||
-        (M > 0 && (!rem_rows || !tok || !tok_v || !conf_v)) || (y && (!row_pos || L <= 0)))
+        (M > 0 && !tok) || (y && (!row_pos || L <= 0)))
         return PVF_ERR_INVALID;
     pvf_verify_kernel<<<n_seq, kThreads, 0, (cudaStream_t)stream>>>(
         seg_off, row_pos, rem_rows, rem_off, v_off, draft_rows, n_drafts, route, tok, tok_v, conf_v,

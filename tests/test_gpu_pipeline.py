@@ -59,19 +59,23 @@ def full_step(ctx, st, flags=0):
 
 
 def verify_pass(ctx, st, sc, cm, sel, osc, ocm, osel, seq_ok, flags=0):
+    """Verification pass laid out from the ORACLE's draft decisions (so that it lines up even when a
+    fragile sequence made the GPU draft differently): the GPU scores it and verifies it with the
+    oracle's selection uploaded; everything is compared sequence by sequence."""
     p = st.params
     prm = params_of(st, flags)
-    if not seq_ok.all():            # decisions differ legitimately somewhere: the layouts would not line up
-        pytest.skip("fragile sequence present")
     v = synth.make_verify_pass(st, osel["rem_rows"], osel["rem_off"], osel["n_drafts"])
     assert np.array_equal(v.v_off, osel["v_off"])
     scv = ctx.score(upload_bits(v.hv_bits))
     seg, pos = t_i32(st.seg_off), t_i32(st.row_pos)
-    ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"])
+    sel_up = dict(rem_rows=t_i32(osel["rem_rows"]), rem_off=t_i32(osel["rem_off"]), v_off=t_i32(osel["v_off"]),
+                  draft_rows=t_i32(osel["draft_rows"]), n_drafts=t_i32(osel["n_drafts"]), route=t_u8(osel["route"]))
+    ver = ctx.verify(prm, seg, pos, sel_up, t_i32(osc["tok"]), scv["tok"], scv["conf"], t_u8(ocm["commit"]))
     torch.cuda.synchronize()
     assert ctx.last_status() == 0
     oscv = oscore.score(st.w_bits, v.hv_bits, st.plan_ids)
-    check_score(to_np(scv), oscv, st.vocab, st.plan_ids)
+    if v.hv_bits.shape[0]:
+        check_score(to_np(scv), oscv, st.vocab, st.plan_ids)
     over = ostep.verify(osc["tok"], ocm["commit"], st.seg_off, st.row_pos, osel["rem_rows"], osel["rem_off"],
                         osel["v_off"], osel["draft_rows"], osel["n_drafts"], osel["route"], oscv["tok"], oscv["conf"],
                         p["tau_high"], p["budget"])
@@ -87,8 +91,8 @@ def verify_pass(ctx, st, sc, cm, sel, osc, ocm, osel, seq_ok, flags=0):
         assert np.array_equal(gv["accept"][b], over["accept"][b]) and gv["choice"][b] == over["choice"][b]
         rows = slice(st.seg_off[b], st.seg_off[b + 1])
         assert np.array_equal(gv["final_commit"][rows], over["final_commit"][rows])
-    assert n_checked >= (st.n_seq + 1) // 2
-    return over
+    assert n_checked >= (st.n_seq + 1) // 2 or st.n_seq == 1
+    return over, n_checked
 
 
 @pytest.mark.parametrize("stress", [False, True])
@@ -109,7 +113,7 @@ def test_config2_and_3_at_small_vocab(stress):
     over = verify_pass(ctx, st2, *full_step(ctx, st2))
     ctx.close()
     st3 = synth.config3(stress=stress, w_bits=w, vocab=8192, hidden=256, n_seq=8, gen_len=128)
-    ctx = make_ctx(w, st3.plan_ids, 8192, 64, 16)
+    ctx = make_ctx(w, st3.plan_ids, 65536, 64, 16)
     verify_pass(ctx, st3, *full_step(ctx, st3))
     ctx.close()
 
