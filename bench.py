@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the fused PVF step on one node.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1a|cfg1b|cfg2|cfg3]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1a|cfg1b|cfg2|cfg3|cfg3s]
 
 A step is one pass of the whole hot path over one synthetic batch, through the C interface:
     pvf_score(H) -> pvf_commit -> pvf_select_drafts -> pvf_score(Hv, verification pass) -> pvf_verify
@@ -55,6 +55,8 @@ def make_workload(name: str, synth, seed_w: int = 1001):
         st = synth.config2(w_bits=w_bits)
     elif name == "cfg3":
         st = synth.config3(w_bits=w_bits)
+    elif name == "cfg3s":                 # 8 of config 3's 64 sequences: the size profiler captures use
+        st = synth.config3(w_bits=w_bits, n_seq=8)
     else:
         raise SystemExit("unknown workload " + name)
     return st
@@ -168,7 +170,7 @@ def run_ours(args):
     p = st.params
     M, V, D = st.n_rows, st.vocab, st.hidden
     K = int(p["budget"])
-    max_rows = 8192 if M <= 4096 else M * (2 + K)       # room for the verification pass
+    max_rows = max(8192, M * (2 + K))                   # room for the verification pass
     ctx = binding.Context(binding.bf16_from_bits(st.w_bits, dev), st.plan_ids, max_rows, max(64, st.n_seq), max(16, K))
     prm = binding.make_params(p["tau_high"], p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], K)
     i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(dev)
@@ -367,7 +369,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg3"])
+    ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg3", "cfg3s"])
     ap.add_argument("--cpu-rows", type=int, default=256, help="rows per pass the CPU baseline scores")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

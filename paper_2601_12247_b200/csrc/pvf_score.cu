@@ -518,7 +518,7 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm)
         const int units_per_block = (g.units + splits - 1) / splits;
         const double t_mma = (double)units_per_block * kUnit * kTileM * 2.0 * D / flops_per_sm;
         const double t_hbm = 2.0 * V * (double)D / hbm;
-        const double cost = waves * (t_mma > t_hbm ? t_mma : t_hbm);
+        const double cost = waves * (t_mma > t_hbm ? t_mma : t_hbm) + waves * t_hbm * 0.25;
         if (best_waves == 0 || cost < best_cost * 0.999) {
             best_cost = cost; best_waves = waves; best_mb = mb; best_splits = splits;
         }
