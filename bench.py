@@ -34,6 +34,12 @@ if ROOT not in sys.path:
 METRIC = "masked positions scored/s per fused PVF step"
 UNIT = "positions/s"
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one GEMM launch, from the ncu captures
+# summarised under profiles/: the config-1a launch was captured as is; larger workloads scale the
+# compute-bound capture (3 passes over W, 13704 rows: 3.636 GB) by their number of passes ("waves").
+NCU_TRAFFIC_CFG1A = 1.0408e9
+NCU_TRAFFIC_PER_WAVE = 3.636e9 / 3
+
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -277,7 +283,11 @@ def run_ours(args):
     else:
         roof = dict(bound="tensor", achieved=alg_flops / t_gemm / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof.update(traffic=None, kernel="pvf_score_gemm_kernel", launches=n_gemm, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
+    if args.workload == "cfg1a":
+        traffic = NCU_TRAFFIC_CFG1A
+    else:
+        traffic = NCU_TRAFFIC_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
+    roof.update(traffic=traffic, kernel="pvf_score_gemm_kernel", launches=n_gemm, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
                 algorithmic_bytes_per_launch=alg_bytes / max(n_gemm, 1), peak_source=peaks["source"] +
                 (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy bandwidth)"))
 
