@@ -1,0 +1,138 @@
+"""Synthetic PVF decode loop on the GPU (Algorithm 1), driving the C interface step by step.
+
+The transformer is replaced by the seeded generator of ``synth``: at every step the hidden states of
+the scored rows are re-drawn on the host from (seed, step, sequence, position), with an amplitude that
+grows with the sequence's committed fraction, and uploaded.  Decoding is semi-autoregressive: the
+working block of a sequence is its first block that still holds a mask; the scored rows are that block's
+masked positions.  One step = draft-pass score, commit, draft selection, verification-pass score, verify;
+it counts as one batched forward.  ``budget = 0`` gives confidence-threshold decoding.
+
+This is a harness around the library (the hot path is the five kernels); it reports steps,
+tokens per forward, scored rows and the kernel time per step measured with CUDA events.
+
+    python -m paper_2601_12247_b200.decode_loop [--n-seq 32] [--gen-len 256] [--block 32] [--budget 4]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+from typing import Callable, Dict, Optional
+
+import numpy as np
+import torch
+
+from . import binding, synth
+
+
+def working_rows(y: np.ndarray, mask_id: int, block: int):
+    """Masked positions of each unfinished sequence's first block that holds a mask."""
+    n_seq, L = y.shape
+    masked = y == mask_id
+    has = masked.any(axis=1)
+    first = np.where(has, masked.argmax(axis=1), 0)
+    blk = first // block
+    pos_grid = np.arange(L)[None, :]
+    in_block = (pos_grid >= (blk * block)[:, None]) & (pos_grid < ((blk + 1) * block)[:, None])
+    take = masked & in_block & has[:, None]
+    seq_ids, positions = np.nonzero(take)                      # row-major: sequences, then ascending position
+    seg_off = np.concatenate([[0], np.cumsum(take.sum(axis=1))]).astype(np.int32)
+    return seq_ids.astype(np.int32), positions.astype(np.int32), seg_off
+
+
+def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: int, gen_len: int, block: int,
+           params: Dict, mask_id: int, max_steps: int = 100000,
+           on_step: Optional[Callable[[int, Dict], None]] = None) -> Dict:
+    """Run the loop until no masks remain.  ``params`` holds tau_high, tau_plan_lo, tau_plan_hi, tau_ar_lo
+    and budget.  Returns y, step counts, scored rows and kernel times."""
+    dev = ctx.device
+    n_seq = targets.shape[0]
+    K = int(params["budget"])
+    prm = binding.make_params(params["tau_high"], params["tau_plan_lo"], params["tau_plan_hi"], params["tau_ar_lo"],
+                              K, binding.PVF_FORCE_PROGRESS)
+    y_dev = torch.full((n_seq, gen_len), mask_id, dtype=torch.int32, device=dev)
+    y = np.full((n_seq, gen_len), mask_id, dtype=np.int32)
+    steps_per_seq = np.zeros(n_seq, dtype=np.int32)
+    scored_rows, n_steps, kernel_ms = 0, 0, 0.0
+    to_dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(dev)
+    while (y == mask_id).any():
+        if n_steps >= max_steps:
+            raise RuntimeError("decode loop did not terminate")
+        seq_ids, positions, seg_off = working_rows(y, mask_id, block)
+        frac = (y != mask_id).sum(axis=1) / float(gen_len)
+        h_bits = synth.loop_hidden(w_bits, targets, seed, n_steps, 0, seq_ids, positions, frac)
+        h = binding.bf16_from_bits(h_bits, dev)
+        seg, pos = to_dev(seg_off, np.int32), to_dev(positions, np.int32)
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        e[0].record()
+        sc = ctx.score(h)
+        cm = ctx.commit(prm, seg, pos, None, sc["tok"], sc["conf"], y=y_dev)
+        sel = ver = scv = None
+        hv_bits = None
+        if K > 0:
+            sel = ctx.select_drafts(prm, seg, pos, None, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
+        e[1].record()
+        scored_rows += len(positions)
+        if K > 0:
+            # the "model forward" of the verification branches: host-side generator
+            s = {k: v.cpu().numpy() for k, v in sel.items()}
+            vb, vi, vc = [], [], []
+            for b in range(n_seq):
+                if s["n_drafts"][b] > 0:
+                    rem = s["rem_rows"][s["rem_off"][b]:s["rem_off"][b + 1]]
+                    for c in range(1 + int(s["n_drafts"][b])):
+                        vb.append(np.full(len(rem), b, np.int32)); vi.append(positions[rem]); vc.append(np.full(len(rem), c, np.int32))
+            cat = lambda l: np.concatenate(l) if l else np.zeros(0, np.int32)
+            vb, vi, vc = cat(vb), cat(vi), cat(vc)
+            hv_bits = synth.loop_verify_hidden(w_bits, targets, seed, n_steps, vb, vi, vc, frac)
+            hv = binding.bf16_from_bits(hv_bits, dev)
+            e[2].record()
+            scv = ctx.score(hv)
+            ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"], y=y_dev)
+            e[3].record()
+            scored_rows += len(vb)
+        torch.cuda.synchronize()
+        kernel_ms += e[0].elapsed_time(e[1]) + (e[2].elapsed_time(e[3]) if K > 0 else 0.0)
+        y = y_dev.cpu().numpy()
+        steps_per_seq += (np.diff(seg_off) > 0).astype(np.int32)
+        if on_step is not None:
+            on_step(n_steps, dict(seq_ids=seq_ids, positions=positions, seg_off=seg_off, h_bits=h_bits, hv_bits=hv_bits,
+                                  score=sc, commit=cm, select=sel, score_v=scv, verify=ver, y=y.copy()))
+        n_steps += 1
+    status = ctx.last_status()
+    return dict(y=y, steps=n_steps, steps_per_seq=steps_per_seq, scored_rows=scored_rows, status=status,
+                tokens_per_forward=float(np.mean(gen_len / np.maximum(steps_per_seq, 1))),
+                kernel_ms_per_step=kernel_ms / max(n_steps, 1), kernel_ms_total=kernel_ms)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--vocab", type=int, default=synth.LLADA_VOCAB)
+    ap.add_argument("--hidden", type=int, default=synth.LLADA_HIDDEN)
+    ap.add_argument("--n-seq", type=int, default=32)
+    ap.add_argument("--gen-len", type=int, default=256)
+    ap.add_argument("--block", type=int, default=32)
+    ap.add_argument("--budget", type=int, default=4)
+    ap.add_argument("--n-plan", type=int, default=2048)
+    ap.add_argument("--q-plan", type=float, default=0.0, help="fraction of targets drawn from the planning ids")
+    ap.add_argument("--seed", type=int, default=1004)
+    args = ap.parse_args()
+    dev = torch.device("cuda:0")
+    w_bits = synth.make_w(args.seed, args.vocab, args.hidden)
+    plan = synth.make_plan_ids(args.seed, args.vocab, args.n_plan)
+    targets = synth.loop_targets(args.seed, args.vocab, args.n_seq, args.gen_len, plan, args.q_plan)
+    ctx = binding.Context(binding.bf16_from_bits(w_bits, dev), plan, args.n_seq * args.block * (2 + args.budget),
+                          args.n_seq, max(args.budget, 1))
+    p = dict(tau_high=0.9, budget=args.budget, **synth.DEFAULT_BAND)
+    out = {}
+    for name, budget in (("pvf", args.budget), ("threshold_only", 0)):
+        r = decode(ctx, w_bits, targets, args.seed, args.gen_len, args.block, dict(p, budget=budget), args.vocab - 128)
+        out[name] = dict(steps=r["steps"], mean_steps_per_sequence=float(r["steps_per_seq"].mean()),
+                         tokens_per_forward=r["tokens_per_forward"], scored_rows=r["scored_rows"],
+                         kernel_ms_per_step=r["kernel_ms_per_step"], status=r["status"])
+    out["config"] = dict(vocab=args.vocab, hidden=args.hidden, n_seq=args.n_seq, gen_len=args.gen_len, block=args.block,
+                         budget=args.budget, q_plan=args.q_plan, data="synthetic")
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

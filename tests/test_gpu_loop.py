@@ -1,0 +1,103 @@
+"""Config 4: the synthetic decode loop on the GPU against the oracle's loop, state by state."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import loop as oloop
+from oracle import score as oscore
+from paper_2601_12247_b200 import binding, decode_loop, synth
+from gpu_util import FRAGILE, NEAR_TIE, check_score, dev, make_ctx, to_np
+
+
+def test_working_rows_matches_oracle_rule():
+    rng = np.random.default_rng(0)
+    for _ in range(20):
+        y = rng.integers(0, 50, (5, 64)).astype(np.int32)
+        y[rng.random((5, 64)) < 0.5] = 99
+        y[0] = 3                                             # a finished sequence
+        a = decode_loop.working_rows(y, 99, 16)
+        b = oloop.working_rows(y, 99, 16)
+        for u, v in zip(a, b):
+            assert np.array_equal(u, v)
+
+
+def fragile_step(h, p):
+    """True if the oracle's step holds a row whose decision could legitimately flip on the GPU."""
+    def bad(sc, taus):
+        f = sc["gap"] < NEAR_TIE
+        for t in taus:
+            f |= np.abs(sc["conf"] - float(np.float32(t))) < FRAGILE
+        return bool(f.any())
+    return bad(h["score"], [p["tau_high"], p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"]])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("budget,q_plan", [(4, 0.5), (0, 0.0), (3, 0.0)])
+def test_loop_tiny_shape_state_by_state(budget, q_plan):
+    V, D, B, L, S, seed = 4096, 256, 4, 64, 32, 1004
+    w = synth.make_w(seed, V, D)
+    plan = synth.make_plan_ids(seed, V, 256)
+    tg = synth.loop_targets(seed, V, B, L, plan, q_plan)
+    p = dict(tau_high=0.9, budget=budget, **synth.DEFAULT_BAND)
+    mask = V - 1
+    want = oloop.decode(synth, w, plan, tg, seed, L, S, p, mask, trace=True)
+    ctx = make_ctx(w, plan, B * S * (2 + budget), B, max(budget, 1))
+    trace = []
+    got = decode_loop.decode(ctx, w, tg, seed, L, S, p, mask, on_step=lambda s, d: trace.append(d))
+    assert got["status"] == 0
+    n_same = 0
+    for s, (g, o) in enumerate(zip(trace, want["history"])):
+        if fragile_step(o, p):
+            break
+        assert np.array_equal(g["positions"], o["positions"]) and np.array_equal(g["seq_ids"], o["seq_ids"])
+        check_score(to_np(g["score"]), o["score"], V, plan)
+        assert np.array_equal(to_np(g["commit"])["commit"], o["commit"]["commit"])
+        if budget > 0:
+            gs, os_ = to_np(g["select"]), o["select"]
+            for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+                assert np.array_equal(gs[k], os_[k]), (s, k)
+            if os_["v_off"][-1] > 0:
+                osv = oscore.score(w, g["hv_bits"], plan)
+                if (osv["gap"] < NEAR_TIE).any() or (np.abs(osv["conf"] - float(np.float32(0.9))) < FRAGILE).any():
+                    break
+                gv = to_np(g["verify"])
+                for k in ("accept", "choice", "final_commit"):
+                    assert np.array_equal(gv[k], o["verify"][k]), (s, k)
+        assert np.array_equal(g["y"], o["y"]), s
+        n_same += 1
+    assert n_same >= min(5, want["steps"])
+    if n_same == want["steps"]:
+        assert got["steps"] == want["steps"] and np.array_equal(got["y"], want["y"])
+        assert np.array_equal(got["steps_per_seq"], want["steps_per_seq"])
+    # invariants that hold whatever happened
+    assert not (got["y"] == mask).any()
+    prev = np.full((B, L), mask, np.int32)
+    for g in trace:
+        keep = prev != mask
+        assert np.array_equal(g["y"][keep], prev[keep])
+        prev = g["y"]
+    ctx.close()
+
+
+@pytest.mark.gpu
+def test_loop_llada_shape_two_sequences_sampled_rows():
+    # full vocabulary and hidden size, short canvas: every step's scores are checked on sampled rows
+    V, D, B, L, S, seed = synth.LLADA_VOCAB, synth.LLADA_HIDDEN, 2, 32, 16, 1004
+    w = synth.make_w(seed, V, D)
+    plan = synth.make_plan_ids(seed, V, 2048)
+    tg = synth.loop_targets(seed, V, B, L, plan, 0.5)
+    p = dict(tau_high=0.9, budget=4, **synth.DEFAULT_BAND)
+    ctx = make_ctx(w, plan, 4096, B, 4)
+    checked = []
+
+    def on_step(s, d):
+        if s < 3 and len(d["positions"]):
+            rows = np.unique(np.linspace(0, len(d["positions"]) - 1, 3).astype(int))
+            check_score(to_np(d["score"]), oscore.score(w, d["h_bits"][rows], plan), V, plan, rows=rows)
+            checked.append(s)
+
+    got = decode_loop.decode(ctx, w, tg, seed, L, S, p, V - 128, on_step=on_step)
+    assert got["status"] == 0 and not (got["y"] == V - 128).any() and len(checked) >= 2
+    base = decode_loop.decode(ctx, w, tg, seed, L, S, dict(p, budget=0), V - 128)
+    assert got["steps_per_seq"].sum() <= base["steps_per_seq"].sum() + 2
+    ctx.close()
