@@ -119,7 +119,7 @@ def main():
     dev = torch.device("cuda:0")
     w_bits = synth.make_w(args.seed, args.vocab, args.hidden)
     plan = synth.make_plan_ids(args.seed, args.vocab, args.n_plan)
-    targets = synth.loop_targets(args.seed, args.vocab, args.n_seq, args.gen_len, plan, args.q_plan)
+    targets = synth.loop_targets(args.seed, args.vocab, args.n_seq, args.gen_len, plan, args.q_plan, avoid=args.vocab - 128)
     ctx = binding.Context(binding.bf16_from_bits(w_bits, dev), plan, args.n_seq * args.block * (2 + args.budget),
                           args.n_seq, max(args.budget, 1))
     p = dict(tau_high=0.9, budget=args.budget, **synth.DEFAULT_BAND)

@@ -304,8 +304,10 @@ def make_verify_pass(step: StepInputs, rem_rows: np.ndarray, rem_off: np.ndarray
 
 
 def loop_targets(seed: int, vocab: int, n_seq: int, gen_len: int, plan_ids: Optional[np.ndarray] = None,
-                 q_plan: float = 0.0) -> np.ndarray:
-    """Target token of every (sequence, position) of the decode loop; fixed across steps."""
+                 q_plan: float = 0.0, avoid: Optional[int] = None) -> np.ndarray:
+    """Target token of every (sequence, position) of the decode loop; fixed across steps.  A target
+    equal to ``avoid`` (the mask id: committing it would leave the position masked for ever) is moved
+    to the next id."""
     t = np.empty((n_seq, gen_len), dtype=np.int32)
     for b in range(n_seq):
         for i in range(gen_len):
@@ -314,6 +316,8 @@ def loop_targets(seed: int, vocab: int, n_seq: int, gen_len: int, plan_ids: Opti
                 gp = _rng(seed, TAG_PLAN_PICK, b, i)
                 if gp.random() < q_plan:
                     v = int(plan_ids[int(gp.integers(0, len(plan_ids)))])
+            if avoid is not None and v == avoid:
+                v = (v + 1) % vocab
             t[b, i] = v
     return t
 

@@ -37,7 +37,7 @@ def test_loop_tiny_shape_state_by_state(budget, q_plan):
     V, D, B, L, S, seed = 4096, 256, 4, 64, 32, 1004
     w = synth.make_w(seed, V, D)
     plan = synth.make_plan_ids(seed, V, 256)
-    tg = synth.loop_targets(seed, V, B, L, plan, q_plan)
+    tg = synth.loop_targets(seed, V, B, L, plan, q_plan, avoid=V - 1)
     p = dict(tau_high=0.9, budget=budget, **synth.DEFAULT_BAND)
     mask = V - 1
     want = oloop.decode(synth, w, plan, tg, seed, L, S, p, mask, trace=True)
@@ -85,7 +85,7 @@ def test_loop_llada_shape_two_sequences_sampled_rows():
     V, D, B, L, S, seed = synth.LLADA_VOCAB, synth.LLADA_HIDDEN, 2, 32, 16, 1004
     w = synth.make_w(seed, V, D)
     plan = synth.make_plan_ids(seed, V, 2048)
-    tg = synth.loop_targets(seed, V, B, L, plan, 0.5)
+    tg = synth.loop_targets(seed, V, B, L, plan, 0.5, avoid=V - 128)
     p = dict(tau_high=0.9, budget=4, **synth.DEFAULT_BAND)
     ctx = make_ctx(w, plan, 4096, B, 4)
     checked = []

@@ -14,7 +14,7 @@ MASK = V - 1
 def setup():
     w = synth.make_w(SEED, V, D)
     plan = synth.make_plan_ids(SEED, V, 128)
-    tg = synth.loop_targets(SEED, V, B, L, plan, 0.5)
+    tg = synth.loop_targets(SEED, V, B, L, plan, 0.5, avoid=MASK)
     return w, plan, tg
 
 
