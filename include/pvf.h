@@ -49,7 +49,8 @@ enum {
     PVF_ERR_UNSUPPORTED = -3, /* device is not sm_100, or a shape outside what the kernels handle */
     PVF_ERR_CUDA = -4,        /* a CUDA runtime or driver call failed */
     PVF_ERR_TIMEOUT = -5,     /* (status word only) a bounded wait inside a kernel ran out */
-    PVF_ERR_WORKSPACE = -6    /* workspace too small or not 256-byte aligned */
+    PVF_ERR_WORKSPACE = -6,   /* workspace too small or not 256-byte aligned */
+    PVF_ERR_TOO_LARGE = -7    /* pvf_score_static only: more rows than its built-in scratch array holds */
 };
 
 /* Limits of a context.  max_rows bounds M of every call, max_seqs bounds n_seq, max_budget bounds K. */
@@ -191,6 +192,46 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
                const int32_t *tok, const int32_t *tok_v, const float *conf_v, const uint8_t *commit,
                uint8_t *accept, int32_t *choice, uint8_t *final_commit,
                int32_t *y, int32_t L, void *stream);
+
+/*
+ * pvf_score_static -- pvf_score for callers that must not allocate.  (The paper has no counterpart: this
+ * is a packaging variant of pvf_score, same arithmetic, same kernels.)
+ *
+ * Some callers of this library cannot call cudaMalloc at the point where they score: code that runs
+ * inside a memory-pool or arena discipline where every device byte is accounted for up front, plugins
+ * loaded into a host process that forbids allocation after start-up, and latency-critical serving loops
+ * where an allocation (and the implicit device synchronisation it can cause) is not acceptable.  pvf_score
+ * asks such callers for a workspace through pvf_create; this entry point needs neither a context nor a
+ * workspace.  Its scratch memory -- the per-vocabulary-range softmax states that the GEMM kernel writes and
+ * the merge kernel reads -- is a fixed 512.25 KiB array inside the library image.  Every GPU that loads
+ * the library holds that array until the process exits, whether or not this function is ever called.
+ *
+ *   w_head       device, bf16 [vocab][hidden_size] row-major, 16-byte aligned
+ *   hidden       device, bf16 [M][hidden_size], 16-byte aligned; hidden_size a multiple of 8
+ *   M            at most PVF_STATIC_MAX_ROWS; larger M returns PVF_ERR_TOO_LARGE and launches nothing
+ *   plan_bitmap  device, ceil(vocab/32) words, bit v set iff token v is in P^plan; may be NULL when
+ *                in_plan is NULL
+ *   tok, conf, ent, in_plan   outputs as in pvf_score (ent and in_plan may be NULL)
+ *
+ * The call itself allocates nothing: no cudaMalloc / cudaFree, no allocating library routine; it
+ * encodes three tensor maps on the host, clears one status word with cudaMemsetAsync and launches the two
+ * scoring kernels on `stream`.  The first call on each device additionally looks up the array's device
+ * address and raises the GEMM kernel's shared-memory limit (this also makes the CUDA runtime load the
+ * kernels); make that first call with the device current and before any stream capture begins.
+ *
+ * All calls on a device share the one array, and it keeps the last call's contents.  Only the status word
+ * has to start from zero and the call clears it; the softmax states are fully rewritten before they are
+ * read.  Two calls that overlap on the GPU (different streams without an ordering between them, or two
+ * threads) race on the array and give wrong results: serialise them.
+ *
+ * pvf_score_static_status copies the status word of the current device to *status (PVF_OK or
+ * PVF_ERR_TIMEOUT of the most recent call); it synchronises the device.
+ */
+#define PVF_STATIC_MAX_ROWS 1024
+int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, const void *hidden, int32_t M,
+                     const uint32_t *plan_bitmap, int32_t *tok, float *conf, float *ent, uint8_t *in_plan,
+                     void *stream);
+int pvf_score_static_status(int32_t *status);
 
 #ifdef __cplusplus
 }

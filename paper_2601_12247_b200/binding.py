@@ -18,6 +18,8 @@ LIB_PATH = os.path.join(_HERE, "libpvf.so")
 
 PVF_OK = 0
 PVF_ERR_INVALID, PVF_ERR_ALIGN, PVF_ERR_UNSUPPORTED, PVF_ERR_CUDA, PVF_ERR_TIMEOUT, PVF_ERR_WORKSPACE = -1, -2, -3, -4, -5, -6
+PVF_ERR_TOO_LARGE = -7
+PVF_STATIC_MAX_ROWS = 1024
 PVF_FORCE_PROGRESS = 1
 PVF_EXCLUDE_SELF_FROM_IMPACT = 2
 
@@ -64,6 +66,8 @@ def load() -> ctypes.CDLL:
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
         lib.pvf_verify.argtypes = [vp, pp, i32, i32] + [vp] * 16 + [i32, vp]; lib.pvf_verify.restype = ctypes.c_int
+        lib.pvf_score_static.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]; lib.pvf_score_static.restype = ctypes.c_int
+        lib.pvf_score_static_status.argtypes = [ctypes.POINTER(i32)]; lib.pvf_score_static_status.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -215,3 +219,26 @@ def bf16_from_bits(bits: np.ndarray, device) -> torch.Tensor:
     """uint16 bf16 bit patterns (numpy) -> torch.bfloat16 tensor on `device`."""
     t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
     return t.to(device).view(torch.bfloat16)
+
+
+def score_static(w_head: torch.Tensor, hidden: torch.Tensor, out: Dict[str, torch.Tensor],
+                 plan_bitmap: Optional[torch.Tensor] = None) -> int:
+    """pvf_score_static: scoring without a context or workspace, for callers that cannot allocate.
+
+    Everything is passed in: ``out`` holds the preallocated tok / conf (and optionally ent, in_plan)
+    tensors, ``plan_bitmap`` an optional int32 device tensor of ceil(V/32) words.  Returns the C return
+    code (PVF_OK, or e.g. PVF_ERR_TOO_LARGE above PVF_STATIC_MAX_ROWS rows) instead of raising, and
+    allocates nothing itself.  Calls that overlap on the GPU race on the library's built-in scratch
+    array; make the first call on a device before any stream capture."""
+    lib = load()
+    V, D = w_head.shape
+    return int(lib.pvf_score_static(_ptr(w_head), V, D, _ptr(hidden), hidden.shape[0], _ptr(plan_bitmap),
+                                    _ptr(out["tok"]), _ptr(out["conf"]), _ptr(out.get("ent")), _ptr(out.get("in_plan")),
+                                    _stream()))
+
+
+def score_static_status() -> int:
+    """Status word of the most recent pvf_score_static call on the current device (synchronises)."""
+    st = ctypes.c_int32()
+    _check(load().pvf_score_static_status(ctypes.byref(st)), "pvf_score_static_status")
+    return int(st.value)

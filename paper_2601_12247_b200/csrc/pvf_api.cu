@@ -62,6 +62,7 @@ const char *pvf_strerror(int code)
         case PVF_ERR_CUDA: return "CUDA call failed";
         case PVF_ERR_TIMEOUT: return "a bounded wait inside a kernel ran out";
         case PVF_ERR_WORKSPACE: return "workspace too small or misaligned";
+        case PVF_ERR_TOO_LARGE: return "more rows than the built-in scratch array of pvf_score_static holds";
         default: return "unknown error";
     }
 }

@@ -610,3 +610,109 @@ int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------- pvf_score_static
+// Scoring for callers that cannot allocate: the per-range softmax states (the only scratch the scoring
+// kernels need) live in a fixed array inside the library image instead of a caller-provided workspace.
+namespace {
+
+constexpr int kStaticMaxRows = PVF_STATIC_MAX_ROWS;
+constexpr int kStaticMaxSms = 256;                              // head-room over today's 148 SMs
+constexpr size_t kStaticHeaderBytes = 256;                      // status word, padded
+constexpr size_t kStaticPartialsBytes = (size_t)kTileM * kStaticMaxSms * sizeof(float4);
+constexpr int kStaticMaxDevices = 64;
+
+// Every GPU that loads this library holds these 512.25 KiB until the process exits.
+static __device__ __align__(256) unsigned char pvf_static_scratch[kStaticHeaderBytes + kStaticPartialsBytes];
+
+struct StaticDeviceState {
+    bool ready;
+    int n_sm;
+    unsigned char *scratch;     // device address of pvf_static_scratch on that GPU
+};
+StaticDeviceState g_static_state[kStaticMaxDevices];
+
+// Once per device, with that device current: resolve the array's device address (its name is only a
+// host-side handle here) and raise the GEMM kernel's shared-memory limit.
+int static_device_state(StaticDeviceState **out)
+{
+    int device = 0, cc = 0, n_sm = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return PVF_ERR_CUDA;
+    if (device < 0 || device >= kStaticMaxDevices) return PVF_ERR_UNSUPPORTED;
+    StaticDeviceState *st = &g_static_state[device];
+    if (!st->ready) {
+        if (cudaDeviceGetAttribute(&cc, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+            return PVF_ERR_CUDA;
+        if (cc != 10 || n_sm > kStaticMaxSms) return PVF_ERR_UNSUPPORTED;
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, pvf_static_scratch) != cudaSuccess || !ptr) return PVF_ERR_CUDA;
+        if (cudaFuncSetAttribute(pvf_score_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return PVF_ERR_CUDA;
+        st->scratch = (unsigned char *)ptr;
+        st->n_sm = n_sm;
+        st->ready = true;
+    }
+    *out = st;
+    return PVF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, const void *hidden, int32_t M,
+                     const uint32_t *plan_bitmap, int32_t *tok, float *conf, float *ent, uint8_t *in_plan,
+                     void *stream)
+{
+    if (vocab <= 0 || hidden_size <= 0 || M < 0) return PVF_ERR_INVALID;
+    if (M > kStaticMaxRows) return PVF_ERR_TOO_LARGE;
+    if (M == 0) return PVF_OK;
+    if (!w_head || !hidden || !tok || !conf || (in_plan && !plan_bitmap)) return PVF_ERR_INVALID;
+    if (hidden_size % 8 != 0 || ((uintptr_t)w_head & 15) != 0 || ((uintptr_t)hidden & 15) != 0) return PVF_ERR_ALIGN;
+    StaticDeviceState *st = nullptr;
+    int rc = static_device_state(&st);
+    if (rc != PVF_OK) return rc;
+    const pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden_size, st->n_sm);
+    if ((size_t)M * g.splits * sizeof(float4) > kStaticPartialsBytes) return PVF_ERR_TOO_LARGE;
+
+    CUtensorMap tm_h, tm_w_full, tm_w_unit;
+    if ((rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)hidden_size, (uint32_t)g.a_rows)) != PVF_OK) return rc;
+    if ((rc = make_tensor_map(&tm_w_full, w_head, (uint64_t)vocab, (uint64_t)hidden_size, kTileN)) != PVF_OK) return rc;
+    if ((rc = make_tensor_map(&tm_w_unit, w_head, (uint64_t)vocab, (uint64_t)hidden_size, kUnit)) != PVF_OK) return rc;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    int32_t *status = (int32_t *)st->scratch;
+    float4 *partials = (float4 *)(st->scratch + kStaticHeaderBytes);
+    // The array keeps the previous call's contents.  The status word must start at zero; the partial
+    // states need no clearing: the GEMM kernel writes every (row, range) entry the merge kernel reads.
+    if (cudaMemsetAsync(status, 0, sizeof(int32_t), s) != cudaSuccess) return PVF_ERR_CUDA;
+
+    ScoreArgs a;
+    a.M = M; a.V = vocab; a.D = hidden_size;
+    a.num_kb = (hidden_size + kBlockK - 1) / kBlockK;
+    a.units = g.units;
+    a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
+    a.a_rows = g.a_rows;
+    a.partials = partials;
+    a.status = status;
+    pvf_score_gemm_kernel<<<g.ctas, kThreads, kSmemBytes, s>>>(tm_h, tm_w_full, tm_w_unit, a);
+    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
+    const int warps_per_block = 8;
+    pvf_score_merge_kernel<<<(M + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(
+        partials, M, g.splits, plan_bitmap, tok, conf, ent, in_plan);
+    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
+    return PVF_OK;
+}
+
+int pvf_score_static_status(int32_t *status)
+{
+    if (!status) return PVF_ERR_INVALID;
+    StaticDeviceState *st = nullptr;
+    int rc = static_device_state(&st);
+    if (rc != PVF_OK) return rc;
+    if (cudaMemcpy(status, st->scratch, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return PVF_ERR_CUDA;
+    return PVF_OK;
+}
+
+}  // extern "C"
