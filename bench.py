@@ -113,6 +113,24 @@ class ClockSampler:
                     samples=len(sm), power_w_max=float(max(power)))
 
 
+def max_over_ranks(ms: float, device=None) -> float:
+    """Slowest rank's elapsed time (all-reduce MAX over the default process group; identity when
+    torch.distributed is not initialised)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(rows_per_rank: int, steps: int, ms: float, world: int) -> float:
+    """Rows all ranks processed divided by the slowest rank's time (replicas: every rank does the
+    same work on its own batch)."""
+    return world * rows_per_rank * steps / (ms * 1e-3)
+
+
 # ------------------------------------------------------------------------------------ reference arm
 def run_reference(args):
     """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
@@ -260,14 +278,9 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop()
     ctx.set_score_events(None, None)
-    ms = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1), dev)
     status = ctx.last_status()
-    value = world * M * args.steps / (ms * 1e-3)
+    value = whole_job_value(M, args.steps, ms, world)
 
     # roofline of the dominant kernel (the score GEMM), from the events recorded in the timed region
     gemm_ms = sum(a.elapsed_time(b) for a, b, _ in ev_pairs)
@@ -291,45 +304,36 @@ def run_ours(args):
                 algorithmic_bytes_per_launch=alg_bytes / max(n_gemm, 1), peak_source=peaks["source"] +
                 (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy bandwidth)"))
 
-    # ---------------- end to end: inputs start in pinned host memory, results end in host memory
+    # ---------------- end to end: the host-buffer C entry points (inputs in pinned host memory, every
+    # result copied back to host memory, stream synchronised inside each call)
     n_e2e = max(3, min(args.steps, 200))
-    host_out = {k: torch.empty(v.shape, dtype=v.dtype).pin_memory() for k, v in
-                dict(tok=o_sc["tok"], conf=o_sc["conf"], commit=o_cm["commit"], draft_rows=o_sel["draft_rows"],
-                     n_drafts=o_sel["n_drafts"], route=o_sel["route"], v_off=o_sel["v_off"], accept=o_ver["accept"],
-                     choice=o_ver["choice"], final_commit=o_ver["final_commit"]).items()}
-    h_dev2 = torch.empty_like(h)
-    hv_dev2 = torch.empty_like(hv) if Mv else None
+    ctx.attach_host_staging()
+    hb = binding.host_buffers(M, st.n_seq, K, Mv)
+    seg_h = torch.from_numpy(np.ascontiguousarray(st.seg_off, dtype=np.int32)).pin_memory()
+    pos_h = torch.from_numpy(np.ascontiguousarray(st.row_pos, dtype=np.int32)).pin_memory()
+    act_h = torch.from_numpy(np.ascontiguousarray(st.active)).pin_memory()
 
     def e2e_step():
-        h_dev2.copy_(h_host, non_blocking=True)
-        if Mv:
-            hv_dev2.copy_(hv_host, non_blocking=True)
-        step(h_dev2, hv_dev2)
-        for k, src in (("tok", o_sc["tok"]), ("conf", o_sc["conf"]), ("commit", o_cm["commit"]),
-                       ("draft_rows", o_sel["draft_rows"]), ("n_drafts", o_sel["n_drafts"]), ("route", o_sel["route"]),
-                       ("v_off", o_sel["v_off"]), ("accept", o_ver["accept"]), ("choice", o_ver["choice"]),
-                       ("final_commit", o_ver["final_commit"])):
-            host_out[k].copy_(src, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        ctx.draft_step_host(prm, h_host, seg_h, pos_h, act_h, hb)
+        ctx.verify_step_host(prm, hv_host, hb)
 
     for _ in range(3):
         e2e_step()
+    if int(hb["v_off"][-1]) != Mv:
+        raise SystemExit("host-buffer step laid out %d verification rows, expected %d" % (int(hb["v_off"][-1]), Mv))
     barrier()
     e0.record()
     for _ in range(n_e2e):
         e2e_step()
     e1.record()
     barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    h2d = int(h_host.numel() * 2 + (hv_host.numel() * 2 if Mv else 0))
-    d2h = int(sum(v.numel() * v.element_size() for v in host_out.values()))
-    e2e = dict(value=world * M * n_e2e / (ms_e2e * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
-               steps=n_e2e, ms_per_step=ms_e2e / n_e2e)
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), dev)
+    h2d = int(h_host.numel() * 2 + (hv_host.numel() * 2 if Mv else 0) + seg_h.numel() * 4 + pos_h.numel() * 4 + act_h.numel())
+    d2h_keys_draft = ("tok", "conf", "ent", "in_plan", "commit", "draft_rows", "n_drafts", "route", "rem_off", "v_off")
+    d2h = int(sum(hb[k].numel() * hb[k].element_size() for k in d2h_keys_draft) + M * 4        # rem_rows: M entries
+              + Mv * 8 + hb["accept"].numel() + hb["choice"].numel() * 4 + M)
+    e2e = dict(value=whole_job_value(M, n_e2e, ms_e2e, world), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+               steps=n_e2e, ms_per_step=ms_e2e / n_e2e, api="pvf_draft_step_host + pvf_verify_step_host")
 
     # ---------------- CPU baseline: the oracle on the same step (rank 0, single-GPU runs only)
     cpu = None

@@ -194,6 +194,34 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
                int32_t *y, int32_t L, void *stream);
 
 /*
+ * Host-buffer variants of the step (Algorithm 1, one decoding iteration split at the model's
+ * verification forward).  Every array argument is a HOST pointer (pinned memory makes the copies
+ * asynchronous); the library copies inputs into a device staging buffer, runs the device entry points
+ * above on `stream`, copies the results back and synchronises the stream before returning.  Output
+ * pointers may be NULL (that result is not copied back).
+ *
+ *   pvf_host_staging_bytes   bytes of device staging a context of this shape needs (about
+ *                            max_rows * (2 * hidden + 40) bytes)
+ *   pvf_attach_host_staging  hand the context a 256-byte-aligned device buffer of that size (kept until
+ *                            replaced; NULL detaches).  Without it the two calls return PVF_ERR_WORKSPACE.
+ *   pvf_draft_step_host      pvf_score + pvf_commit + pvf_select_drafts on hidden_host[M][hidden]; outputs
+ *                            as in those calls.  The device copies stay in the staging buffer.
+ *   pvf_verify_step_host     pvf_score on hidden_v_host[Mv][hidden] + pvf_verify, continuing the draft
+ *                            half most recently run on this context (same budget); Mv must equal that
+ *                            half's v_off[n_seq].
+ */
+size_t pvf_host_staging_bytes(const pvf_shape *shape);
+int pvf_attach_host_staging(pvf_ctx *ctx, void *staging, size_t bytes);
+int pvf_draft_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hidden_host, int32_t M, int32_t n_seq,
+                        const int32_t *seg_off_host, const int32_t *row_pos_host, const uint8_t *active_host,
+                        int32_t *tok_host, float *conf_host, float *ent_host, uint8_t *in_plan_host,
+                        uint8_t *commit_host, int32_t *draft_rows_host, int32_t *n_drafts_host, uint8_t *route_host,
+                        int32_t *rem_rows_host, int32_t *rem_off_host, int32_t *v_off_host, void *stream);
+int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hidden_v_host, int32_t Mv,
+                         int32_t *tok_v_host, float *conf_v_host, uint8_t *accept_host, int32_t *choice_host,
+                         uint8_t *final_commit_host, void *stream);
+
+/*
  * pvf_score_static -- pvf_score for callers that must not allocate.  (The paper has no counterpart: this
  * is a packaging variant of pvf_score, same arithmetic, same kernels.)
  *

@@ -66,6 +66,10 @@ def load() -> ctypes.CDLL:
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
         lib.pvf_verify.argtypes = [vp, pp, i32, i32] + [vp] * 16 + [i32, vp]; lib.pvf_verify.restype = ctypes.c_int
+        lib.pvf_host_staging_bytes.argtypes = [ps]; lib.pvf_host_staging_bytes.restype = sz
+        lib.pvf_attach_host_staging.argtypes = [vp, vp, sz]; lib.pvf_attach_host_staging.restype = ctypes.c_int
+        lib.pvf_draft_step_host.argtypes = [vp, pp, vp, i32, i32] + [vp] * 14 + [vp]; lib.pvf_draft_step_host.restype = ctypes.c_int
+        lib.pvf_verify_step_host.argtypes = [vp, pp, vp, i32] + [vp] * 5 + [vp]; lib.pvf_verify_step_host.restype = ctypes.c_int
         lib.pvf_score_static.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]; lib.pvf_score_static.restype = ctypes.c_int
         lib.pvf_score_static_status.argtypes = [ctypes.POINTER(i32)]; lib.pvf_score_static_status.restype = ctypes.c_int
         _lib = lib
@@ -153,6 +157,35 @@ class Context:
         _check(self.lib.pvf_score_plan(self.handle, int(M), *[ctypes.byref(x) for x in v]), "pvf_score_plan")
         return dict(ctas=v[0].value, splits=v[1].value, waves=v[2].value, launches=v[3].value)
 
+    # ------------------------------------------------------------------ host-buffer variants
+    def attach_host_staging(self):
+        """Allocate the device staging buffer of the host-buffer calls and hand it to the context."""
+        nbytes = self.lib.pvf_host_staging_bytes(ctypes.byref(self.shape))
+        self.staging = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        off = (-self.staging.data_ptr()) % 256
+        _check(self.lib.pvf_attach_host_staging(self.handle, ctypes.c_void_p(self.staging.data_ptr() + off), nbytes),
+               "pvf_attach_host_staging")
+
+    def draft_step_host(self, params: pvf_params, hidden_host: torch.Tensor, seg_off: torch.Tensor, row_pos: torch.Tensor,
+                        active: Optional[torch.Tensor], out: Dict[str, torch.Tensor]):
+        """pvf_draft_step_host: all tensors are CPU tensors; returns after the results are in ``out``."""
+        hp = lambda k: _ptr(out.get(k))
+        rc = self.lib.pvf_draft_step_host(self.handle, ctypes.byref(params), _ptr(hidden_host), hidden_host.shape[0],
+                                          seg_off.shape[0] - 1, _ptr(seg_off), _ptr(row_pos), _ptr(active),
+                                          hp("tok"), hp("conf"), hp("ent"), hp("in_plan"), hp("commit"), hp("draft_rows"),
+                                          hp("n_drafts"), hp("route"), hp("rem_rows"), hp("rem_off"), hp("v_off"), _stream())
+        _check(rc, "pvf_draft_step_host")
+        return out
+
+    def verify_step_host(self, params: pvf_params, hidden_v_host: Optional[torch.Tensor], out: Dict[str, torch.Tensor]):
+        """pvf_verify_step_host: continues the last draft_step_host of this context."""
+        Mv = 0 if hidden_v_host is None else hidden_v_host.shape[0]
+        hp = lambda k: _ptr(out.get(k))
+        rc = self.lib.pvf_verify_step_host(self.handle, ctypes.byref(params), _ptr(hidden_v_host), Mv,
+                                           hp("tok_v"), hp("conf_v"), hp("accept"), hp("choice"), hp("final_commit"), _stream())
+        _check(rc, "pvf_verify_step_host")
+        return out
+
     # ------------------------------------------------------------------ the four calls
     def score(self, hidden: torch.Tensor, out: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, torch.Tensor]:
         assert hidden.is_cuda and hidden.dtype == torch.bfloat16 and hidden.is_contiguous()
@@ -213,6 +246,16 @@ class Context:
                                  _ptr(y), L, _stream())
         _check(rc, "pvf_verify")
         return out
+
+
+def host_buffers(M: int, n_seq: int, budget: int, Mv: int = 0, pinned: bool = True) -> Dict[str, torch.Tensor]:
+    """Host tensors (pinned by default) for every output of the host-buffer step calls."""
+    mk = lambda shape, dt: (torch.empty(shape, dtype=dt).pin_memory() if pinned else torch.empty(shape, dtype=dt))
+    return dict(tok=mk(M, torch.int32), conf=mk(M, torch.float32), ent=mk(M, torch.float32), in_plan=mk(M, torch.uint8),
+                commit=mk(M, torch.uint8), draft_rows=mk((n_seq, budget), torch.int32), n_drafts=mk(n_seq, torch.int32),
+                route=mk(n_seq, torch.uint8), rem_rows=mk(max(M, 1), torch.int32), rem_off=mk(n_seq + 1, torch.int32),
+                v_off=mk(n_seq + 1, torch.int32), tok_v=mk(max(Mv, 1), torch.int32), conf_v=mk(max(Mv, 1), torch.float32),
+                accept=mk((n_seq, budget), torch.uint8), choice=mk(n_seq, torch.int32), final_commit=mk(M, torch.uint8))
 
 
 def bf16_from_bits(bits: np.ndarray, device) -> torch.Tensor:

@@ -106,6 +106,10 @@ int pvf_create(pvf_ctx **out, const pvf_shape *shape, const void *w_head,
     ctx->partials_bytes = l.partials_bytes;
     ctx->ev_start = nullptr;
     ctx->ev_stop = nullptr;
+    ctx->staging = nullptr;
+    ctx->staging_bytes = 0;
+    ctx->host_rows = ctx->host_seqs = ctx->host_budget = 0;
+    ctx->host_active = false;
 
     std::vector<uint32_t> bitmap(l.bitmap_bytes / 4, 0u);
     for (int32_t i = 0; i < n_plan; ++i) bitmap[plan_ids_host[i] >> 5] |= 1u << (plan_ids_host[i] & 31);

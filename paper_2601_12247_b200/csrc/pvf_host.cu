@@ -1,0 +1,157 @@
+// Host-buffer variants of the step: inputs and outputs live in host memory, the library stages them
+// through a caller-provided device buffer with cudaMemcpyAsync and synchronises the stream before
+// returning.  The arithmetic is the device entry points' (pvf_score, pvf_commit, pvf_select_drafts,
+// pvf_verify); nothing is computed on the host.
+#include "pvf_internal.h"
+
+namespace {
+
+struct StagingLayout {
+    size_t hidden, seg_off, row_pos, active, tok, conf, ent, in_plan, commit, n_commit, draft_rows, n_drafts,
+        route, rem_rows, rem_off, v_off, tok_v, conf_v, accept, choice, final_commit, total;
+};
+
+StagingLayout staging_layout(const pvf_shape *s)
+{
+    StagingLayout l;
+    size_t off = 0;
+    const size_t R = (size_t)s->max_rows, B = (size_t)s->max_seqs, K = (size_t)(s->max_budget > 0 ? s->max_budget : 1);
+    auto take = [&](size_t bytes) { size_t o = off; off = pvf_align_up(off + bytes, 256); return o; };
+    l.hidden = take(R * (size_t)s->hidden * 2);
+    l.seg_off = take((B + 1) * 4);
+    l.row_pos = take(R * 4);
+    l.active = take(R);
+    l.tok = take(R * 4);
+    l.conf = take(R * 4);
+    l.ent = take(R * 4);
+    l.in_plan = take(R);
+    l.commit = take(R);
+    l.n_commit = take(B * 4);
+    l.draft_rows = take(B * K * 4);
+    l.n_drafts = take(B * 4);
+    l.route = take(B);
+    l.rem_rows = take(R * 4 + 4);
+    l.rem_off = take((B + 1) * 4);
+    l.v_off = take((B + 1) * 4);
+    l.tok_v = take(R * 4);
+    l.conf_v = take(R * 4);
+    l.accept = take(B * K);
+    l.choice = take(B * 4);
+    l.final_commit = take(R);
+    l.total = off;
+    return l;
+}
+
+bool h2d(void *dst, const void *src, size_t n, cudaStream_t s)
+{
+    return n == 0 || cudaMemcpyAsync(dst, src, n, cudaMemcpyHostToDevice, s) == cudaSuccess;
+}
+bool d2h(void *dst, const void *src, size_t n, cudaStream_t s)
+{
+    return n == 0 || !dst || cudaMemcpyAsync(dst, src, n, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t pvf_host_staging_bytes(const pvf_shape *shape)
+{
+    if (!shape || shape->vocab <= 0 || shape->hidden <= 0 || shape->max_rows < 0 || shape->max_seqs < 0 ||
+        shape->max_budget < 0)
+        return 0;
+    return staging_layout(shape).total;
+}
+
+int pvf_attach_host_staging(pvf_ctx *ctx, void *staging, size_t bytes)
+{
+    if (!ctx) return PVF_ERR_INVALID;
+    if (!staging) { ctx->staging = nullptr; ctx->staging_bytes = 0; return PVF_OK; }
+    if (((uintptr_t)staging & 255) != 0 || bytes < staging_layout(&ctx->shape).total) return PVF_ERR_WORKSPACE;
+    ctx->staging = (uint8_t *)staging;
+    ctx->staging_bytes = bytes;
+    ctx->host_rows = 0;
+    ctx->host_seqs = 0;
+    return PVF_OK;
+}
+
+int pvf_draft_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hidden_host, int32_t M, int32_t n_seq,
+                        const int32_t *seg_off_host, const int32_t *row_pos_host, const uint8_t *active_host,
+                        int32_t *tok_host, float *conf_host, float *ent_host, uint8_t *in_plan_host,
+                        uint8_t *commit_host, int32_t *draft_rows_host, int32_t *n_drafts_host, uint8_t *route_host,
+                        int32_t *rem_rows_host, int32_t *rem_off_host, int32_t *v_off_host, void *stream)
+{
+    if (!ctx || !params || M < 0 || n_seq < 0 || M > ctx->shape.max_rows || n_seq > ctx->shape.max_seqs ||
+        params->budget < 0 || params->budget > ctx->shape.max_budget)
+        return PVF_ERR_INVALID;
+    if (!ctx->staging) return PVF_ERR_WORKSPACE;
+    if (M == 0 || n_seq == 0) { ctx->host_rows = 0; ctx->host_seqs = 0; return (M == 0) ? PVF_OK : PVF_ERR_INVALID; }
+    if (!hidden_host || !seg_off_host || !row_pos_host) return PVF_ERR_INVALID;
+    const StagingLayout l = staging_layout(&ctx->shape);
+    uint8_t *g = ctx->staging;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t K = (size_t)params->budget;
+    const uint8_t *active_dev = active_host ? g + l.active : nullptr;
+    if (!h2d(g + l.hidden, hidden_host, (size_t)M * ctx->shape.hidden * 2, s) ||
+        !h2d(g + l.seg_off, seg_off_host, ((size_t)n_seq + 1) * 4, s) ||
+        !h2d(g + l.row_pos, row_pos_host, (size_t)M * 4, s) ||
+        (active_host && !h2d(g + l.active, active_host, (size_t)M, s)))
+        return PVF_ERR_CUDA;
+    int rc = pvf_score(ctx, g + l.hidden, M, (int32_t *)(g + l.tok), (float *)(g + l.conf), (float *)(g + l.ent),
+                       g + l.in_plan, stream);
+    if (rc != PVF_OK) return rc;
+    rc = pvf_commit(ctx, params, M, n_seq, (const int32_t *)(g + l.seg_off), (const int32_t *)(g + l.row_pos), active_dev,
+                    (const int32_t *)(g + l.tok), (const float *)(g + l.conf), g + l.commit, (int32_t *)(g + l.n_commit),
+                    nullptr, 0, stream);
+    if (rc != PVF_OK) return rc;
+    rc = pvf_select_drafts(ctx, params, M, n_seq, (const int32_t *)(g + l.seg_off), (const int32_t *)(g + l.row_pos),
+                           active_dev, (const int32_t *)(g + l.tok), (const float *)(g + l.conf), g + l.in_plan,
+                           g + l.commit, (int32_t *)(g + l.draft_rows), (int32_t *)(g + l.n_drafts), g + l.route,
+                           (int32_t *)(g + l.rem_rows), (int32_t *)(g + l.rem_off), (int32_t *)(g + l.v_off), stream);
+    if (rc != PVF_OK) return rc;
+    const bool ok = d2h(tok_host, g + l.tok, (size_t)M * 4, s) && d2h(conf_host, g + l.conf, (size_t)M * 4, s) &&
+                    d2h(ent_host, g + l.ent, (size_t)M * 4, s) && d2h(in_plan_host, g + l.in_plan, (size_t)M, s) &&
+                    d2h(commit_host, g + l.commit, (size_t)M, s) &&
+                    d2h(draft_rows_host, g + l.draft_rows, (size_t)n_seq * K * 4, s) &&
+                    d2h(n_drafts_host, g + l.n_drafts, (size_t)n_seq * 4, s) && d2h(route_host, g + l.route, (size_t)n_seq, s) &&
+                    d2h(rem_rows_host, g + l.rem_rows, (size_t)M * 4, s) &&
+                    d2h(rem_off_host, g + l.rem_off, ((size_t)n_seq + 1) * 4, s) &&
+                    d2h(v_off_host, g + l.v_off, ((size_t)n_seq + 1) * 4, s);
+    if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return PVF_ERR_CUDA;
+    ctx->host_rows = M;
+    ctx->host_seqs = n_seq;
+    ctx->host_budget = params->budget;
+    ctx->host_active = active_host != nullptr;
+    return PVF_OK;
+}
+
+int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hidden_v_host, int32_t Mv,
+                         int32_t *tok_v_host, float *conf_v_host, uint8_t *accept_host, int32_t *choice_host,
+                         uint8_t *final_commit_host, void *stream)
+{
+    if (!ctx || !params || Mv < 0 || Mv > ctx->shape.max_rows) return PVF_ERR_INVALID;
+    if (!ctx->staging) return PVF_ERR_WORKSPACE;
+    const int32_t M = ctx->host_rows, n_seq = ctx->host_seqs;
+    if (M <= 0 || n_seq <= 0 || params->budget != ctx->host_budget) return PVF_ERR_INVALID;   // no draft half to continue
+    if (Mv > 0 && !hidden_v_host) return PVF_ERR_INVALID;
+    const StagingLayout l = staging_layout(&ctx->shape);
+    uint8_t *g = ctx->staging;
+    cudaStream_t s = (cudaStream_t)stream;
+    const size_t K = (size_t)params->budget;
+    if (!h2d(g + l.hidden, hidden_v_host, (size_t)Mv * ctx->shape.hidden * 2, s)) return PVF_ERR_CUDA;
+    int rc = pvf_score(ctx, g + l.hidden, Mv, (int32_t *)(g + l.tok_v), (float *)(g + l.conf_v), nullptr, nullptr, stream);
+    if (rc != PVF_OK) return rc;
+    rc = pvf_verify(ctx, params, M, n_seq, (const int32_t *)(g + l.seg_off), (const int32_t *)(g + l.row_pos),
+                    (const int32_t *)(g + l.rem_rows), (const int32_t *)(g + l.rem_off), (const int32_t *)(g + l.v_off),
+                    (const int32_t *)(g + l.draft_rows), (const int32_t *)(g + l.n_drafts), g + l.route,
+                    (const int32_t *)(g + l.tok), (const int32_t *)(g + l.tok_v), (const float *)(g + l.conf_v), g + l.commit,
+                    g + l.accept, (int32_t *)(g + l.choice), g + l.final_commit, nullptr, 0, stream);
+    if (rc != PVF_OK) return rc;
+    const bool ok = d2h(tok_v_host, g + l.tok_v, (size_t)Mv * 4, s) && d2h(conf_v_host, g + l.conf_v, (size_t)Mv * 4, s) &&
+                    d2h(accept_host, g + l.accept, (size_t)n_seq * K, s) && d2h(choice_host, g + l.choice, (size_t)n_seq * 4, s) &&
+                    d2h(final_commit_host, g + l.final_commit, (size_t)M, s);
+    if (!ok || cudaStreamSynchronize(s) != cudaSuccess) return PVF_ERR_CUDA;
+    return PVF_OK;
+}
+
+}  // extern "C"

@@ -31,6 +31,10 @@ struct pvf_ctx {
     CUtensorMap tm_w_full;  // W as [V][D], box 256 rows x 64 columns, 128-byte swizzle
     CUtensorMap tm_w_unit;  // same tensor, box 16 rows x 64 columns
     cudaEvent_t ev_start, ev_stop;   // optional timing hook around the GEMM kernel
+    uint8_t *staging;                // optional device staging of the host-buffer entry points
+    size_t staging_bytes;
+    int32_t host_rows, host_seqs, host_budget;   // shape of the draft half the staging currently holds
+    bool host_active;
 };
 
 // Work split of pvf_score for M rows on n_sm SMs (see pvf_score.cu).
