@@ -9,6 +9,7 @@
 #include "pvf.h"
 
 #define PVF_MAX_BUDGET_LIMIT 64
+#define PVF_W_BOX_LEVELS 5
 
 // Device scalars at the head of the workspace.
 struct pvf_device_words {
@@ -28,8 +29,7 @@ struct pvf_ctx {
     uint32_t *plan_bitmap;  // ceil(V/32) words, bit v set iff v in P^plan
     float4 *partials;       // [rows][splits] per-range softmax states of pvf_score
     size_t partials_bytes;
-    CUtensorMap tm_w_full;  // W as [V][D], box 256 rows x 64 columns, 128-byte swizzle
-    CUtensorMap tm_w_unit;  // same tensor, box 16 rows x 64 columns
+    CUtensorMap tm_w[PVF_W_BOX_LEVELS];   // W as [V][D], boxes of 16 << level rows x 64 columns, 128-byte swizzle
     cudaEvent_t ev_start, ev_stop;   // optional timing hook around the GEMM kernel
     uint8_t *staging;                // optional device staging of the host-buffer entry points
     size_t staging_bytes;
@@ -46,10 +46,42 @@ struct pvf_score_geometry {
     int waves;       // ceil(m_tiles / mb)
     int ctas;        // mb * splits
     int a_rows;      // rows of the hidden-state TMA box
+    int streaming;   // 1: at most 32 rows, handled by the swapped-operand streaming kernel
 };
 pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm);
 size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm);
 int pvf_score_init(pvf_ctx *ctx);   // tensor maps of W, kernel attributes
+
+// Programmatic dependent launch.  Every kernel of the library is launched with pvf_launch and runs
+//     <set-up that touches no global memory>; pvf_launch_dependents(); pvf_grid_dependency_wait();
+// before its first global access, on every thread.  The wait returns once the kernel before it in
+// the stream has completed and its writes are visible, so stream order is kept; what overlaps is the
+// launch latency and set-up of a kernel with the tail of its predecessor.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pvf_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pvf_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t pvf_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+#ifdef PVF_NO_PDL
+    cfg.numAttrs = 0;
+#else
+    cfg.numAttrs = 1;
+#endif
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
 
 static inline size_t pvf_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

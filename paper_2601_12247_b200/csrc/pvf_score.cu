@@ -9,17 +9,19 @@
 // block sweeps a contiguous vocabulary range.  Each (row, range) pair leaves one 16-byte partial
 // state; a small second kernel merges the partials of a row.
 //
-// Thread block = 6 warps:  warp 0 issues TMA loads (W and H tiles, 128-byte swizzle, 4 stages),
-// warp 1 owns tensor memory and issues the MMAs, warps 2-5 are the softmax epilogue.  The two
-// 256-column accumulators alternate, so the epilogue of one vocabulary tile overlaps the MMAs of
-// the next.
+// Thread block = 6 warps:  warp 0 issues TMA loads (W and H tiles, 128-byte swizzle, a ring of
+// stages), warp 1 owns tensor memory and issues the MMAs, warps 2-5 are the softmax epilogue.  Two
+// accumulators alternate, so the epilogue of one vocabulary tile overlaps the MMAs of the next.
+//
+// The GEMM kernel is a template over its tile shape (GemmCfg): vocabulary entries per accumulator,
+// 64-element k-panels per pipeline stage, stages.  Calls with at most 32 rows take a second kernel
+// with the operands swapped (pvf_score_stream_kernel, below): vocabulary on the lanes, rows on the
+// columns, so that no tensor work is spent on padding rows.
 //
 // Work split.  Rows form tiles of 128, the vocabulary granules of 16 entries.  `mb` row tiles are
 // in flight at once, each swept by `splits` blocks over disjoint vocabulary ranges (mb * splits
 // <= number of SMs); blocks that share a range stream the same W tiles at the same time, so W is
 // read from HBM once per wave, and the wave's H tiles stay L2-resident.
-//   M <= 128:  one row tile, one range per SM (pure weight streaming)
-//   M large:   waves of up to 64 row tiles
 //
 // Every wait on an mbarrier is bounded: when one runs out the block records PVF_ERR_TIMEOUT in
 // the status word, raises a block-wide abort flag, drains its outstanding copies and MMAs with
@@ -28,33 +30,78 @@
 
 #include "pvf_internal.h"
 
+// Tile shapes (overridable at build time for tuning sweeps).
+#ifndef PVF_STREAM_STAGES
+#define PVF_STREAM_STAGES 6
+#endif
+#ifndef PVF_GENERAL_TILE_N
+#define PVF_GENERAL_TILE_N 256
+#endif
+#ifndef PVF_GENERAL_PANELS
+#define PVF_GENERAL_PANELS 1
+#endif
+#ifndef PVF_GENERAL_STAGES
+#define PVF_GENERAL_STAGES 4
+#endif
+#ifndef PVF_L2_PROMOTION
+#define PVF_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+#endif
+#ifndef PVF_GEMM_EARLY_TRIGGER
+#define PVF_GEMM_EARLY_TRIGGER 0 // 1: the GEMM kernel releases its dependents before its main loop
+#endif
+#ifndef PVF_W_EVICT_FIRST
+#define PVF_W_EVICT_FIRST 0      // 1: W tiles carry an evict-first L2 hint (they are never re-read)
+#endif
+
 namespace {
 
 constexpr int kTileM = 128;                // rows per accumulator (tensor-memory lanes)
-constexpr int kTileN = 256;                // vocabulary entries per accumulator (columns)
 constexpr int kUnit = 16;                  // vocabulary granule
-constexpr int kBlockK = 64;                // bf16 per k-block = one 128-byte swizzle row
-constexpr int kStages = 4;
-constexpr int kABytes = kTileM * kBlockK * 2;          // 16 KiB
-constexpr int kBBytes = kTileN * kBlockK * 2;          // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kUnitBytes = kUnit * kBlockK * 2;        // 2 KiB
+constexpr int kBlockK = 64;                // bf16 per k-panel = one 128-byte swizzle row
+constexpr int kRowBytes = kBlockK * 2;     // 128
+constexpr int kUnitBytes = kUnit * kRowBytes;          // 2 KiB
 constexpr int kThreads = 192;
 constexpr int kEpilogueThreads = 128;
-constexpr int kTmemCols = 512;
+constexpr int kMaxStages = 16;
+constexpr int kStreamRows = 32;            // the streaming kernel handles at most this many rows
+constexpr int kWBoxLevels = PVF_W_BOX_LEVELS;           // W boxes of 16, 32, 64, 128 and 256 vocabulary entries
 constexpr int kMaxConcurrentTiles = 64;    // cap on the wave's L2-resident H tiles
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
+template <int TILE_N, int PANELS, int STAGES>
+struct GemmCfg {
+    static constexpr int kTileN = TILE_N;              // vocabulary entries per accumulator (columns)
+    static constexpr int kPanels = PANELS;             // 64-element k-panels per stage
+    static constexpr int kStages = STAGES;
+    static constexpr int kAPanelBytes = kTileM * kRowBytes;
+    static constexpr int kBPanelBytes = TILE_N * kRowBytes;
+    static constexpr int kStageBytes = PANELS * (kAPanelBytes + kBPanelBytes);
+    static constexpr int kUnitsPerTile = TILE_N / kUnit;
+    static constexpr int kTmemCols = 2 * TILE_N;
+    static constexpr int kControlBytes = 512;
+    static constexpr int kSmemBytes = STAGES * kStageBytes + 1024 /*alignment slack*/ + kControlBytes;
+    static_assert(TILE_N == 64 || TILE_N == 128 || TILE_N == 256, "accumulator width");
+    static_assert(STAGES >= 2 && STAGES <= kMaxStages, "stages");
+    static_assert(kSmemBytes <= 227 * 1024, "shared memory");
+};
+
+using GeneralCfg = GemmCfg<PVF_GENERAL_TILE_N, PVF_GENERAL_PANELS, PVF_GENERAL_STAGES>;
+
 struct __align__(8) SharedControl {
-    unsigned long long full[kStages];      // TMA bytes landed
-    unsigned long long empty[kStages];     // MMAs that read the stage have completed
+    unsigned long long full[kMaxStages];   // TMA bytes landed
+    unsigned long long empty[kMaxStages];  // MMAs that read the stage have completed
     unsigned long long acc_full[2];        // accumulator complete
     unsigned long long acc_empty[2];       // epilogue has drained the accumulator
     unsigned long long drain;              // abort path: all issued MMAs completed
     uint32_t tmem_base;
     volatile int abort_flag;
 };
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*control*/;
+static_assert(sizeof(SharedControl) <= 512, "control block");
+
+// W as [V][D] seen through boxes of 16 << level rows x 64 columns.
+struct WMaps {
+    CUtensorMap level[kWBoxLevels];
+};
 
 struct ScoreArgs {
     int M, V, D;
@@ -125,6 +172,22 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y) : "memory");
 }
+#if PVF_W_EVICT_FIRST
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y,
+                                                 unsigned long long policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+__device__ __forceinline__ unsigned long long l2_evict_first_policy()
+{
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+#endif
 
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -193,6 +256,31 @@ __device__ __forceinline__ void split_range(int units, int splits, int q, int *u
     *u1 = (int)((long long)units * (q + 1) / splits);
 }
 
+// Vocabulary tiles of a range of `range` granules starting at u0.  A short range (up to
+// kBalanceMaxTiles tiles) is cut into near-equal tiles: with full tiles plus a small ragged one, the
+// ragged tile's pipeline stages would hold too few bytes to keep HBM busy, and in the weight-streaming
+// regime that tile is a tenth of the block's work.  A long range keeps full tiles (one TMA box each).
+constexpr int kBalanceMaxTiles = 16;
+struct TileSplit {
+    int u0, range, n_tiles, units_per_tile;
+    bool balanced;
+    __device__ __forceinline__ TileSplit(int u0_, int u1_, int units_per_tile_)
+        : u0(u0_), range(u1_ - u0_), n_tiles((u1_ - u0_ + units_per_tile_ - 1) / units_per_tile_),
+          units_per_tile(units_per_tile_), balanced(n_tiles <= kBalanceMaxTiles) {}
+    // first granule and number of granules of tile t
+    __device__ __forceinline__ void tile(int t, int *tu0, int *tun) const
+    {
+        if (balanced) {
+            const int a = range * t / n_tiles, b = range * (t + 1) / n_tiles;
+            *tu0 = u0 + a;
+            *tun = b - a;
+        } else {
+            *tu0 = u0 + t * units_per_tile;
+            *tun = min(units_per_tile, u0 + range - *tu0);
+        }
+    }
+};
+
 // Running softmax state of one row over the columns seen so far.
 struct RowState {
     float m;      // running max
@@ -234,16 +322,46 @@ __device__ __forceinline__ void fold16(RowState &st, const uint32_t (&raw)[16], 
     }
 }
 
-// ---------------------------------------------------------------------------------- GEMM kernel
-__global__ void __launch_bounds__(kThreads, 1)
-pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_w_full,
-                      const __grid_constant__ CUtensorMap tm_w_unit, const ScoreArgs args)
+// One W tile of `tun` granules starting at granule tu0, columns x .. x+63, into b_dst: the fewest
+// boxes that cover it (a full tile is one box, a ragged one the binary expansion of its size).
+#if PVF_W_EVICT_FIRST
+#define PVF_W_LOAD(dst, level_, row) tma_load_2d_hint(dst, &maps.level[level_], full, x, row, policy)
+#else
+#define PVF_W_LOAD(dst, level_, row) tma_load_2d(dst, &maps.level[level_], full, x, row)
+#endif
+template <int kUnitsPerTile>
+__device__ __forceinline__ void load_w_tile(uint32_t b_dst, const WMaps &maps, uint32_t full, int x, int tu0, int tun,
+                                            unsigned long long policy)
 {
+    (void)policy;
+    constexpr int kTop = kUnitsPerTile == 16 ? 4 : (kUnitsPerTile == 8 ? 3 : 2);
+    if (tun == kUnitsPerTile) {
+        PVF_W_LOAD(b_dst, kTop, tu0 * kUnit);
+        return;
+    }
+    int u = 0;
+    if (kUnitsPerTile > 8 && (tun & 8)) { PVF_W_LOAD(b_dst + u * kUnitBytes, 3, (tu0 + u) * kUnit); u += 8; }
+    if (kUnitsPerTile > 4 && (tun & 4)) { PVF_W_LOAD(b_dst + u * kUnitBytes, 2, (tu0 + u) * kUnit); u += 4; }
+    if (tun & 2) { PVF_W_LOAD(b_dst + u * kUnitBytes, 1, (tu0 + u) * kUnit); u += 2; }
+    if (tun & 1) { PVF_W_LOAD(b_dst + u * kUnitBytes, 0, (tu0 + u) * kUnit); }
+}
+#undef PVF_W_LOAD
+
+// ---------------------------------------------------------------------------------- GEMM kernel
+template <class Cfg>
+__global__ void __launch_bounds__(kThreads, 1)
+pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ WMaps tm_w, const ScoreArgs args)
+{
+    constexpr int kStages = Cfg::kStages;
+    constexpr int kPanels = Cfg::kPanels;
+    constexpr int kTileN = Cfg::kTileN;
+    constexpr int kUnitsPerTile = Cfg::kUnitsPerTile;
+
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;           // swizzled tiles need 1024-byte alignment
     uint8_t *tiles_ptr = smem_raw + (tiles_addr - raw_addr);
-    SharedControl *ctl = reinterpret_cast<SharedControl *>(tiles_ptr + kStages * kStageBytes);
+    SharedControl *ctl = reinterpret_cast<SharedControl *>(tiles_ptr + kStages * Cfg::kStageBytes);
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -251,7 +369,9 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     const int q = blockIdx.x / args.mb;
     int u0, u1;
     split_range(args.units, args.splits, q, &u0, &u1);
-    const int n_tiles = (u1 - u0 + (kTileN / kUnit) - 1) / (kTileN / kUnit);   // vocabulary tiles per sweep
+    const TileSplit split(u0, u1, kUnitsPerTile);
+    const int n_tiles = split.n_tiles;                                   // vocabulary tiles per sweep
+    const int k_steps = (args.num_kb + kPanels - 1) / kPanels;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -267,9 +387,15 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
+#pragma unroll
+        for (int l = 0; l < kWBoxLevels; ++l)
+            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.level[l]) : "memory");
+    }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&ctl->tmem_base)), "r"(kTmemCols) : "memory");
+                     ::"r"(smem_u32(&ctl->tmem_base)), "r"(Cfg::kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before_sync();
@@ -277,12 +403,21 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
 
+    // Everything above touched no global memory: it may overlap the tail of the kernel before this
+    // one in the stream.  From here on the hidden states are read and the partial states written.
+#if PVF_GEMM_EARLY_TRIGGER
+    pvf_launch_dependents();
+#endif
+    pvf_grid_dependency_wait();
+
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w_full) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w_unit) : "memory");
+#if PVF_W_EVICT_FIRST
+            const unsigned long long policy = l2_evict_first_policy();
+#else
+            const unsigned long long policy = 0ull;
+#endif
             int stage = 0;
             uint32_t phase = 0;
             int armed_parity[kStages];
@@ -293,22 +428,22 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
                 const int m_tile = w * args.mb + mt_local;
                 if (m_tile >= args.m_tiles) continue;
                 for (int tile = 0; tile < n_tiles && alive; ++tile) {
-                    const int tu0 = u0 + tile * (kTileN / kUnit);
-                    const int tun = min(kTileN / kUnit, u1 - tu0);              // granules in this tile
-                    const uint32_t bytes = (uint32_t)args.a_rows * (kBlockK * 2) + (uint32_t)tun * kUnitBytes;
-                    for (int kb = 0; kb < args.num_kb; ++kb) {
+                    int tu0, tun;                                              // first granule, granules of this tile
+                    split.tile(tile, &tu0, &tun);
+                    const uint32_t panel_bytes = (uint32_t)args.a_rows * kRowBytes + (uint32_t)tun * kUnitBytes;
+                    for (int step = 0; step < k_steps; ++step) {
+                        const int kb0 = step * kPanels;
+                        const int np = min(kPanels, args.num_kb - kb0);
                         if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
                         const uint32_t full = smem_u32(&ctl->full[stage]);
-                        const uint32_t a_dst = tiles_addr + stage * kStageBytes;
-                        const uint32_t b_dst = a_dst + kABytes;
-                        mbar_arrive_expect_tx(full, bytes);
+                        const uint32_t a_base = tiles_addr + stage * Cfg::kStageBytes;
+                        const uint32_t b_base = a_base + kPanels * Cfg::kAPanelBytes;
+                        mbar_arrive_expect_tx(full, panel_bytes * (uint32_t)np);
                         armed_parity[stage] = (int)phase;
-                        tma_load_2d(a_dst, &tm_h, full, kb * kBlockK, m_tile * kTileM);
-                        if (tun == kTileN / kUnit) {
-                            tma_load_2d(b_dst, &tm_w_full, full, kb * kBlockK, tu0 * kUnit);
-                        } else {
-                            for (int u = 0; u < tun; ++u)
-                                tma_load_2d(b_dst + u * kUnitBytes, &tm_w_unit, full, kb * kBlockK, (tu0 + u) * kUnit);
+                        for (int p = 0; p < np; ++p) {
+                            const int x = (kb0 + p) * kBlockK;
+                            tma_load_2d(a_base + p * Cfg::kAPanelBytes, &tm_h, full, x, m_tile * kTileM);
+                            load_w_tile<kUnitsPerTile>(b_base + p * Cfg::kBPanelBytes, tm_w, full, x, tu0, tun, policy);
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
@@ -335,24 +470,29 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
                 const int m_tile = w * args.mb + mt_local;
                 if (m_tile >= args.m_tiles) continue;
                 for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
-                    const int tu0 = u0 + tile * (kTileN / kUnit);
-                    const int tun = min(kTileN / kUnit, u1 - tu0);
+                    int tu0, tun;
+                    split.tile(tile, &tu0, &tun);
                     const uint32_t idesc = instr_desc_bf16(tun * kUnit);
                     const uint32_t buf = tile_count & 1u;
                     const uint32_t acc_phase = (tile_count >> 1) & 1u;
                     if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), acc_phase ^ 1u, ctl, args.status)) { alive = false; break; }
                     tc_fence_after_sync();
                     const uint32_t tmem_d = tmem_base + buf * kTileN;
-                    for (int kb = 0; kb < args.num_kb; ++kb) {
+                    for (int step = 0; step < k_steps; ++step) {
+                        const int kb0 = step * kPanels;
+                        const int np = min(kPanels, args.num_kb - kb0);
                         if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, ctl, args.status)) { alive = false; break; }
                         tc_fence_after_sync();
-                        const uint32_t a_addr = tiles_addr + stage * kStageBytes;
-                        const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
-                        const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kABytes);
+                        const uint32_t a_base = tiles_addr + stage * Cfg::kStageBytes;
+                        const uint32_t b_base = a_base + kPanels * Cfg::kAPanelBytes;
+                        for (int p = 0; p < np; ++p) {
+                            const uint64_t a_desc = smem_desc_k_major_sw128(a_base + p * Cfg::kAPanelBytes);
+                            const uint64_t b_desc = smem_desc_k_major_sw128(b_base + p * Cfg::kBPanelBytes);
 #pragma unroll
-                        for (int k = 0; k < kBlockK / 16; ++k)       // 16 bf16 = 32 bytes further along K
-                            tc_mma_bf16(tmem_d, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc,
-                                        (kb | k) != 0 ? 1u : 0u);
+                            for (int k = 0; k < kBlockK / 16; ++k)       // 16 bf16 = 32 bytes further along K
+                                tc_mma_bf16(tmem_d, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc,
+                                            (step | p | k) != 0 ? 1u : 0u);
+                        }
                         tc_commit(smem_u32(&ctl->empty[stage]));
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
@@ -381,8 +521,8 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
             RowState st;
             st.m = -INFINITY; st.s = 0.f; st.t = 0.f; st.arg = 0x7fffffff;
             for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
-                const int tu0 = u0 + tile * (kTileN / kUnit);
-                const int tun = min(kTileN / kUnit, u1 - tu0);
+                int tu0, tun;
+                split.tile(tile, &tu0, &tun);
                 const uint32_t buf = tile_count & 1u;
                 const uint32_t acc_phase = (tile_count >> 1) & 1u;
                 if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), acc_phase, ctl, args.status)) { alive = false; break; }
@@ -409,9 +549,274 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
 
     tc_fence_before_sync();
     __syncthreads();
+#if !PVF_GEMM_EARLY_TRIGGER
+    // Only now may the next kernel's blocks become resident: while they wait for this grid they would
+    // share the SM with the MMA and epilogue warps.
+    pvf_launch_dependents();
+#endif
     if (warp == 1) {
         tc_fence_after_sync();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(Cfg::kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------- streaming kernel
+// At most 32 scored rows: the call is a pure stream of W through the SMs, and the only thing that
+// matters is to keep HBM busy while spending as little power as possible on everything else (the
+// SM clocks are power-capped in this regime).  Running 32 rows through 128-row MMAs wastes three
+// quarters of the tensor work, so here the operands are swapped: a 128-entry slice of the vocabulary
+// sits on the 128 lanes of the accumulator and the scored rows are its N = 16 or 32 columns,
+//     D[v][m] = sum_k W[v][k] * H[m][k],
+// one 128 x N x 16 MMA per 16 elements of k and vocabulary slice, nothing wasted.  An epilogue thread
+// now owns a vocabulary lane: it keeps one running softmax state per scored row (for the vocabulary
+// entries that passed through its lane) and the block folds the 128 lanes' states once, at the end,
+// through shared memory.  The per-(row, range) partial state it leaves is the GEMM kernel's.
+constexpr int kStreamStages = PVF_STREAM_STAGES;
+constexpr int kStreamTileN = 256;                                   // vocabulary entries per W tile (two 128-lane slices)
+constexpr int kStreamUnitsPerTile = kStreamTileN / kUnit;
+constexpr int kStreamHBytes = kStreamRows * kRowBytes;              // 4 KiB
+constexpr int kStreamWBytes = kStreamTileN * kRowBytes;             // 32 KiB
+constexpr int kStreamStageBytes = kStreamHBytes + kStreamWBytes;
+constexpr int kStreamTmemCols = 128;                                // 2 buffers x 2 slices x 32 columns
+constexpr int kStreamControlBytes = 512;
+constexpr int kStreamSmemBytes = kStreamStages * kStreamStageBytes + 1024 + kStreamControlBytes;
+static_assert(kStreamStages >= 2 && kStreamStages <= kMaxStages && kStreamSmemBytes <= 227 * 1024, "streaming ring");
+// the end-of-block fold reuses the tile ring: 128 lanes x 32 rows x 16 bytes
+static_assert(kStreamStages * kStreamStageBytes >= kTileM * kStreamRows * 16, "fold scratch");
+
+// State (m, s, t, arg) absorbs one more logit x of vocabulary id v.
+__device__ __forceinline__ void state_push(float &m, float &s, float &t, int &arg, float x, int v)
+{
+    constexpr float kLog2e = 1.4426950408889634f;
+    if (x > m) {                                        // strict: ids ascend, so the lowest id keeps a tie
+        const float d = m - x;
+        const float c = (s > 0.f) ? fast_exp2(d * kLog2e) : 0.f;
+        t = (s > 0.f) ? (t + d * s) * c : 0.f;
+        s *= c;
+        m = x;
+        arg = v;
+    }
+    const float d = x - m;
+    const float e = fast_exp2(d * kLog2e);
+    s += e;
+    t = fmaf(d, e, t);
+}
+
+// a <- a merged with b (two states over disjoint vocabulary sets).
+__device__ __forceinline__ void state_merge(float4 &a, const float4 b)
+{
+    constexpr float kLog2e = 1.4426950408889634f;
+    if (!(b.y > 0.f)) return;
+    if (!(a.y > 0.f)) { a = b; return; }
+    const int ia = __float_as_int(a.w), ib = __float_as_int(b.w);
+    const float m = fmaxf(a.x, b.x);
+    const float da = a.x - m, db = b.x - m;
+    const float ca = fast_exp2(da * kLog2e), cb = fast_exp2(db * kLog2e);
+    const int arg = (a.x > b.x) ? ia : ((b.x > a.x) ? ib : min(ia, ib));
+    a.z = (a.z + da * a.y) * ca + (b.z + db * b.y) * cb;
+    a.y = a.y * ca + b.y * cb;
+    a.x = m;
+    a.w = __int_as_float(arg);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ WMaps tm_w, const ScoreArgs args)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+    uint8_t *tiles_ptr = smem_raw + (tiles_addr - raw_addr);
+    SharedControl *ctl = reinterpret_cast<SharedControl *>(tiles_ptr + kStreamStages * kStreamStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int q = blockIdx.x;                                            // one vocabulary range per block
+    int u0, u1;
+    split_range(args.units, args.splits, q, &u0, &u1);
+    const TileSplit split(u0, u1, kStreamUnitsPerTile);
+    const int n_tiles = split.n_tiles;
+    const int n_cols = args.M <= 16 ? 16 : 32;                           // MMA N: scored rows, padded
+    const int k_steps = args.num_kb;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStreamStages; ++s) {
+            mbar_init(smem_u32(&ctl->full[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueThreads);
+        }
+        mbar_init(smem_u32(&ctl->drain), 1);
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
+#pragma unroll
+        for (int l = 0; l < kWBoxLevels; ++l)
+            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.level[l]) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctl->tmem_base)), "r"(kStreamTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+    pvf_grid_dependency_wait();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int armed_parity[kStreamStages];
+#pragma unroll
+            for (int s = 0; s < kStreamStages; ++s) armed_parity[s] = -1;
+            bool alive = true;
+            for (int tile = 0; tile < n_tiles && alive; ++tile) {
+                int tu0, tun;
+                split.tile(tile, &tu0, &tun);
+                const uint32_t bytes = (uint32_t)args.a_rows * kRowBytes + (uint32_t)tun * kUnitBytes;
+                for (int step = 0; step < k_steps; ++step) {
+                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                    const uint32_t full = smem_u32(&ctl->full[stage]);
+                    const uint32_t h_dst = tiles_addr + stage * kStreamStageBytes;
+                    mbar_arrive_expect_tx(full, bytes);
+                    armed_parity[stage] = (int)phase;
+                    tma_load_2d(h_dst, &tm_h, full, step * kBlockK, 0);
+                    load_w_tile<kStreamUnitsPerTile>(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, 0ull);
+                    if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!alive) {
+                for (int s = 0; s < kStreamStages; ++s)
+                    if (armed_parity[s] >= 0) {
+                        const unsigned long long t0 = global_timer_ns();
+                        while (!mbar_try_wait(smem_u32(&ctl->full[s]), (uint32_t)armed_parity[s]) &&
+                               global_timer_ns() - t0 < kWaitLimitNs) {}
+                    }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool alive = true;
+            const uint32_t idesc = instr_desc_bf16(n_cols);
+            for (int tile = 0; tile < n_tiles && alive; ++tile) {
+                int tu0, tun;
+                split.tile(tile, &tu0, &tun);
+                const int n_slices = tun > kTileM / kUnit ? 2 : 1;       // 128-entry vocabulary slices of this tile
+                const uint32_t buf = (uint32_t)tile & 1u;
+                const uint32_t acc_phase = ((uint32_t)tile >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), acc_phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                tc_fence_after_sync();
+                const uint32_t tmem_d = tmem_base + buf * (2 * kStreamRows);
+                for (int step = 0; step < k_steps; ++step) {
+                    if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, ctl, args.status)) { alive = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t h_addr = tiles_addr + stage * kStreamStageBytes;
+                    const uint64_t h_desc = smem_desc_k_major_sw128(h_addr);
+                    for (int sl = 0; sl < n_slices; ++sl) {
+                        // Slice sl = rows sl*128 .. sl*128+127 of the W tile.  A ragged tile's last slice reads
+                        // rows past its end: stale bytes of the same stage, on lanes the epilogue skips.
+                        const uint64_t w_desc = smem_desc_k_major_sw128(h_addr + kStreamHBytes + sl * (kTileM * kRowBytes));
+#pragma unroll
+                        for (int k = 0; k < kBlockK / 16; ++k)
+                            tc_mma_bf16(tmem_d + sl * kStreamRows, w_desc + (uint64_t)(k * 2), h_desc + (uint64_t)(k * 2), idesc,
+                                        (step | k) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(smem_u32(&ctl->empty[stage]));
+                    if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
+                }
+                if (alive) tc_commit(smem_u32(&ctl->acc_full[buf]));
+            }
+            if (!alive) {
+                tc_commit(smem_u32(&ctl->drain));
+                const unsigned long long t0 = global_timer_ns();
+                while (!mbar_try_wait(smem_u32(&ctl->drain), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax epilogue
+        const int quad = warp & 3;
+        const int acc_lane = quad * 32 + lane;                           // this thread's accumulator lane
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        float sm[kStreamRows], ss[kStreamRows], st[kStreamRows];
+        int sa[kStreamRows];
+#pragma unroll
+        for (int i = 0; i < kStreamRows; ++i) { sm[i] = -INFINITY; ss[i] = 0.f; st[i] = 0.f; sa[i] = 0x7fffffff; }
+        bool alive = true;
+        for (int tile = 0; tile < n_tiles && alive; ++tile) {
+            int tu0, tun;
+            split.tile(tile, &tu0, &tun);
+            const int n_slices = tun > kTileM / kUnit ? 2 : 1;
+            const uint32_t buf = (uint32_t)tile & 1u;
+            const uint32_t acc_phase = ((uint32_t)tile >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), acc_phase, ctl, args.status)) { alive = false; break; }
+            tc_fence_after_sync();
+            const int tile_end = min((tu0 + tun) * kUnit, args.V);
+            for (int sl = 0; sl < n_slices; ++sl) {
+                const int v = tu0 * kUnit + sl * kTileM + acc_lane;      // vocabulary id on this lane
+                const bool real = v < tile_end;
+#pragma unroll
+                for (int half = 0; half < kStreamRows / 16; ++half) {
+                    if (half * 16 < n_cols) {                            // block-uniform
+                        uint32_t raw[16];
+                        tmem_ld16(lane_addr + buf * (2 * kStreamRows) + sl * kStreamRows + half * 16, raw);
+                        tmem_ld_wait();
+                        if (real) {
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                state_push(sm[half * 16 + i], ss[half * 16 + i], st[half * 16 + i], sa[half * 16 + i],
+                                           __uint_as_float(raw[i]), v);
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(smem_u32(&ctl->acc_empty[buf]));
+        }
+        // Fold the 128 lanes.  The tile ring is idle now (every copy landed and every MMA that read it
+        // retired before the last accumulator was published), so it serves as scratch [row][lane].
+        if (alive) {
+            float4 *scratch = reinterpret_cast<float4 *>(tiles_ptr);
+#pragma unroll
+            for (int i = 0; i < kStreamRows; ++i)
+                scratch[i * kTileM + acc_lane] = make_float4(sm[i], ss[i], st[i], __int_as_float(sa[i]));
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+        if (alive && !ctl->abort_flag) {
+            // 4 threads per scored row, each folds 32 lanes in lane order, then the 4 fold together
+            const float4 *scratch = reinterpret_cast<const float4 *>(tiles_ptr);
+            const int e = threadIdx.x - 64;                              // 0..127
+            const int row = e >> 2, part = e & 3;
+            float4 acc = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(0x7fffffff));
+            for (int l = 0; l < 32; ++l) state_merge(acc, scratch[row * kTileM + part * 32 + l]);
+            for (int o = 1; o < 4; o <<= 1) {
+                float4 other;
+                other.x = __shfl_xor_sync(0xffffffffu, acc.x, o);
+                other.y = __shfl_xor_sync(0xffffffffu, acc.y, o);
+                other.z = __shfl_xor_sync(0xffffffffu, acc.z, o);
+                other.w = __shfl_xor_sync(0xffffffffu, acc.w, o);
+                state_merge(acc, other);
+            }
+            if (part == 0 && row < args.M) args.partials[(size_t)row * args.splits + q] = acc;
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    pvf_launch_dependents();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kStreamTmemCols) : "memory");
     }
 }
 
@@ -423,6 +828,8 @@ pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int splits,
                        const uint32_t *__restrict__ plan_bitmap, int32_t *__restrict__ tok,
                        float *__restrict__ conf, float *__restrict__ ent, uint8_t *__restrict__ in_plan)
 {
+    pvf_launch_dependents();
+    pvf_grid_dependency_wait();
     const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (row >= M) return;
@@ -491,9 +898,62 @@ int make_tensor_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t 
     cuuint32_t box[2] = {(cuuint32_t)kBlockK, box_rows};
     cuuint32_t elem[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, elem,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, PVF_L2_PROMOTION,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? PVF_OK : PVF_ERR_CUDA;
+}
+
+int make_w_maps(CUtensorMap *levels, const void *w_head, int vocab, int hidden)
+{
+    for (int l = 0; l < kWBoxLevels; ++l) {
+        const int rc = make_tensor_map(&levels[l], w_head, (uint64_t)vocab, (uint64_t)hidden, (uint32_t)(kUnit << l));
+        if (rc != PVF_OK) return rc;
+    }
+    return PVF_OK;
+}
+
+int raise_shared_memory_limits()
+{
+    if (cudaFuncSetAttribute(pvf_score_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kStreamSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(pvf_score_gemm_kernel<GeneralCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             GeneralCfg::kSmemBytes) != cudaSuccess)
+        return PVF_ERR_CUDA;
+    return PVF_OK;
+}
+
+// Launches the GEMM kernel (shape chosen by the geometry) and the merge kernel on `s`.
+int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, int D, const CUtensorMap *w_levels,
+                 float4 *partials, int32_t *status, const uint32_t *plan_bitmap, int32_t *tok, float *conf, float *ent,
+                 uint8_t *in_plan, cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop)
+{
+    CUtensorMap tm_h;
+    int rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)g.a_rows);
+    if (rc != PVF_OK) return rc;
+    WMaps maps;
+    for (int l = 0; l < kWBoxLevels; ++l) maps.level[l] = w_levels[l];
+
+    ScoreArgs a;
+    a.M = M; a.V = V; a.D = D;
+    a.num_kb = (D + kBlockK - 1) / kBlockK;
+    a.units = g.units;
+    a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
+    a.a_rows = g.a_rows;
+    a.partials = partials;
+    a.status = status;
+    const bool timed = ev_start && ev_stop;
+    if (timed && cudaEventRecord(ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
+    cudaError_t e;
+    if (g.streaming)
+        e = pvf_launch(pvf_score_stream_kernel, dim3(g.ctas), dim3(kThreads), kStreamSmemBytes, s, tm_h, maps, a);
+    else
+        e = pvf_launch(pvf_score_gemm_kernel<GeneralCfg>, dim3(g.ctas), dim3(kThreads), GeneralCfg::kSmemBytes, s, tm_h, maps, a);
+    if (e != cudaSuccess) return PVF_ERR_CUDA;
+    if (timed && cudaEventRecord(ev_stop, s) != cudaSuccess) return PVF_ERR_CUDA;
+    const int warps_per_block = 8;
+    e = pvf_launch(pvf_score_merge_kernel, dim3((M + warps_per_block - 1) / warps_per_block), dim3(warps_per_block * 32), 0, s,
+                   (const float4 *)partials, M, g.splits, plan_bitmap, tok, conf, ent, in_plan);
+    return e == cudaSuccess ? PVF_OK : PVF_ERR_CUDA;
 }
 
 }  // namespace
@@ -504,6 +964,7 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm)
     g.m_tiles = (M + kTileM - 1) / kTileM;
     g.units = (V + kUnit - 1) / kUnit;
     g.a_rows = g.m_tiles == 1 ? ((M + 7) / 8) * 8 : kTileM;
+    g.streaming = (g.m_tiles == 1 && M <= kStreamRows) ? 1 : 0;
     if (g.m_tiles == 0) { g.mb = g.splits = g.waves = g.ctas = 0; return g; }
     // Pick the number of waves: cost = waves * max(per-block MMA work, HBM time of one W pass).
     const double flops_per_sm = 1.0e13, hbm = 6.0e12;
@@ -543,13 +1004,9 @@ size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm)
 
 int pvf_score_init(pvf_ctx *ctx)
 {
-    int rc = make_tensor_map(&ctx->tm_w_full, ctx->w_head, (uint64_t)ctx->shape.vocab, (uint64_t)ctx->shape.hidden, kTileN);
+    const int rc = make_w_maps(ctx->tm_w, ctx->w_head, ctx->shape.vocab, ctx->shape.hidden);
     if (rc != PVF_OK) return rc;
-    rc = make_tensor_map(&ctx->tm_w_unit, ctx->w_head, (uint64_t)ctx->shape.vocab, (uint64_t)ctx->shape.hidden, kUnit);
-    if (rc != PVF_OK) return rc;
-    if (cudaFuncSetAttribute(pvf_score_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-        return PVF_ERR_CUDA;
-    return PVF_OK;
+    return raise_shared_memory_limits();
 }
 
 extern "C" {
@@ -583,30 +1040,8 @@ int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
     const int V = ctx->shape.vocab, D = ctx->shape.hidden;
     const pvf_score_geometry g = pvf_score_geometry_for(M, V, D, ctx->n_sm);
     if ((size_t)M * g.splits * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
-
-    CUtensorMap tm_h;
-    int rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)g.a_rows);
-    if (rc != PVF_OK) return rc;
-
-    ScoreArgs a;
-    a.M = M; a.V = V; a.D = D;
-    a.num_kb = (D + kBlockK - 1) / kBlockK;
-    a.units = g.units;
-    a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
-    a.a_rows = g.a_rows;
-    a.partials = ctx->partials;
-    a.status = &ctx->words->status;
-    cudaStream_t s = (cudaStream_t)stream;
-    const bool timed = ctx->ev_start && ctx->ev_stop;
-    if (timed && cudaEventRecord(ctx->ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
-    pvf_score_gemm_kernel<<<g.ctas, kThreads, kSmemBytes, s>>>(tm_h, ctx->tm_w_full, ctx->tm_w_unit, a);
-    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
-    if (timed && cudaEventRecord(ctx->ev_stop, s) != cudaSuccess) return PVF_ERR_CUDA;
-    const int warps_per_block = 8;
-    pvf_score_merge_kernel<<<(M + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(
-        ctx->partials, M, g.splits, ctx->plan_bitmap, tok, conf, ent, in_plan);
-    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
-    return PVF_OK;
+    return launch_score(g, hidden, M, V, D, ctx->tm_w, ctx->partials, &ctx->words->status, ctx->plan_bitmap, tok, conf,
+                        ent, in_plan, (cudaStream_t)stream, ctx->ev_start, ctx->ev_stop);
 }
 
 }  // extern "C"
@@ -633,7 +1068,7 @@ struct StaticDeviceState {
 StaticDeviceState g_static_state[kStaticMaxDevices];
 
 // Once per device, with that device current: resolve the array's device address (its name is only a
-// host-side handle here) and raise the GEMM kernel's shared-memory limit.
+// host-side handle here) and raise the GEMM kernels' shared-memory limit.
 int static_device_state(StaticDeviceState **out)
 {
     int device = 0, cc = 0, n_sm = 0;
@@ -647,8 +1082,7 @@ int static_device_state(StaticDeviceState **out)
         if (cc != 10 || n_sm > kStaticMaxSms) return PVF_ERR_UNSUPPORTED;
         void *ptr = nullptr;
         if (cudaGetSymbolAddress(&ptr, pvf_static_scratch) != cudaSuccess || !ptr) return PVF_ERR_CUDA;
-        if (cudaFuncSetAttribute(pvf_score_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return PVF_ERR_CUDA;
+        if (raise_shared_memory_limits() != PVF_OK) return PVF_ERR_CUDA;
         st->scratch = (unsigned char *)ptr;
         st->n_sm = n_sm;
         st->ready = true;
@@ -676,10 +1110,8 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     const pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden_size, st->n_sm);
     if ((size_t)M * g.splits * sizeof(float4) > kStaticPartialsBytes) return PVF_ERR_TOO_LARGE;
 
-    CUtensorMap tm_h, tm_w_full, tm_w_unit;
-    if ((rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)hidden_size, (uint32_t)g.a_rows)) != PVF_OK) return rc;
-    if ((rc = make_tensor_map(&tm_w_full, w_head, (uint64_t)vocab, (uint64_t)hidden_size, kTileN)) != PVF_OK) return rc;
-    if ((rc = make_tensor_map(&tm_w_unit, w_head, (uint64_t)vocab, (uint64_t)hidden_size, kUnit)) != PVF_OK) return rc;
+    CUtensorMap w_levels[kWBoxLevels];
+    if ((rc = make_w_maps(w_levels, w_head, vocab, hidden_size)) != PVF_OK) return rc;
 
     cudaStream_t s = (cudaStream_t)stream;
     int32_t *status = (int32_t *)st->scratch;
@@ -687,22 +1119,8 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     // The array keeps the previous call's contents.  The status word must start at zero; the partial
     // states need no clearing: the GEMM kernel writes every (row, range) entry the merge kernel reads.
     if (cudaMemsetAsync(status, 0, sizeof(int32_t), s) != cudaSuccess) return PVF_ERR_CUDA;
-
-    ScoreArgs a;
-    a.M = M; a.V = vocab; a.D = hidden_size;
-    a.num_kb = (hidden_size + kBlockK - 1) / kBlockK;
-    a.units = g.units;
-    a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
-    a.a_rows = g.a_rows;
-    a.partials = partials;
-    a.status = status;
-    pvf_score_gemm_kernel<<<g.ctas, kThreads, kSmemBytes, s>>>(tm_h, tm_w_full, tm_w_unit, a);
-    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
-    const int warps_per_block = 8;
-    pvf_score_merge_kernel<<<(M + warps_per_block - 1) / warps_per_block, warps_per_block * 32, 0, s>>>(
-        partials, M, g.splits, plan_bitmap, tok, conf, ent, in_plan);
-    if (cudaGetLastError() != cudaSuccess) return PVF_ERR_CUDA;
-    return PVF_OK;
+    return launch_score(g, hidden, M, vocab, hidden_size, w_levels, partials, status, plan_bitmap, tok, conf, ent,
+                        in_plan, s, nullptr, nullptr);
 }
 
 int pvf_score_static_status(int32_t *status)

@@ -72,6 +72,8 @@ pvf_commit_kernel(const int32_t *__restrict__ seg_off, const int32_t *__restrict
 {
     __shared__ int s_int[kWarps];
     __shared__ unsigned long long s_key[kWarps];
+    pvf_launch_dependents();
+    pvf_grid_dependency_wait();
     const int b = blockIdx.x;
     const int r0 = seg_off[b], r1 = seg_off[b + 1];
     int count = 0;
@@ -117,6 +119,8 @@ pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t 
     __shared__ int s_int[kWarps];
     __shared__ unsigned long long s_key[kWarps];
     __shared__ int s_last;
+    pvf_launch_dependents();
+    pvf_grid_dependency_wait();
     const int b = blockIdx.x;
     const int r0 = seg_off[b], r1 = seg_off[b + 1];
 
@@ -235,6 +239,8 @@ pvf_verify_kernel(const int32_t *__restrict__ seg_off, const int32_t *__restrict
     __shared__ int s_acc[PVF_MAX_BUDGET_LIMIT];
     __shared__ double s_c[PVF_MAX_BUDGET_LIMIT];
     __shared__ int s_choice;
+    pvf_launch_dependents();
+    pvf_grid_dependency_wait();
     const int b = blockIdx.x;
     const int r0 = seg_off[b], r1 = seg_off[b + 1];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -335,9 +341,9 @@ bool params_ok(const pvf_ctx *ctx, const pvf_params *p, int32_t M, int32_t n_seq
            p->budget >= 0 && p->budget <= ctx->shape.max_budget;
 }
 
-int launch_result()
+int launch_result(cudaError_t e)
 {
-    return cudaGetLastError() == cudaSuccess ? PVF_OK : PVF_ERR_CUDA;
+    return e == cudaSuccess ? PVF_OK : PVF_ERR_CUDA;
 }
 
 }  // namespace
@@ -352,10 +358,9 @@ int pvf_commit(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
     if (!params_ok(ctx, params, M, n_seq)) return PVF_ERR_INVALID;
     if (n_seq == 0) return M == 0 ? PVF_OK : PVF_ERR_INVALID;
     if (!seg_off || !conf || !commit || (M > 0 && y && (!row_pos || !tok || L <= 0))) return PVF_ERR_INVALID;
-    pvf_commit_kernel<<<n_seq, kThreads, 0, (cudaStream_t)stream>>>(
-        seg_off, row_pos, active, tok, conf, params->tau_high,
-        (params->flags & PVF_FORCE_PROGRESS) ? 1 : 0, commit, n_commit, y, L);
-    return launch_result();
+    return launch_result(pvf_launch(pvf_commit_kernel, dim3(n_seq), dim3(kThreads), 0, (cudaStream_t)stream,
+                                    seg_off, row_pos, active, tok, conf, params->tau_high,
+                                    (params->flags & PVF_FORCE_PROGRESS) ? 1 : 0, commit, n_commit, y, L));
 }
 
 int pvf_select_drafts(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
@@ -371,11 +376,10 @@ int pvf_select_drafts(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t
     if (!seg_off || !conf || !in_plan || !commit || !n_drafts || !route || !rem_off || !v_off ||
         (params->budget > 0 && !draft_rows) || (M > 0 && !rem_rows))
         return PVF_ERR_INVALID;
-    pvf_select_kernel<<<n_seq, kThreads, 0, (cudaStream_t)stream>>>(
-        n_seq, seg_off, active, conf, in_plan, commit, params->tau_plan_lo, params->tau_plan_hi,
-        params->tau_ar_lo, params->budget, draft_rows, n_drafts, route, rem_rows, rem_off, v_off,
-        &ctx->words->select_ticket);
-    return launch_result();
+    return launch_result(pvf_launch(pvf_select_kernel, dim3(n_seq), dim3(kThreads), 0, (cudaStream_t)stream,
+                                    n_seq, seg_off, active, conf, in_plan, commit, params->tau_plan_lo,
+                                    params->tau_plan_hi, params->tau_ar_lo, params->budget, draft_rows, n_drafts,
+                                    route, rem_rows, rem_off, v_off, &ctx->words->select_ticket));
 }
 
 int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
@@ -392,11 +396,11 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
         (params->budget > 0 && (!draft_rows || !accept)) ||
         (M > 0 && !tok) || (y && (!row_pos || L <= 0)))
         return PVF_ERR_INVALID;
-    pvf_verify_kernel<<<n_seq, kThreads, 0, (cudaStream_t)stream>>>(
-        seg_off, row_pos, rem_rows, rem_off, v_off, draft_rows, n_drafts, route, tok, tok_v, conf_v,
-        commit, params->tau_high, params->budget, (params->flags & PVF_EXCLUDE_SELF_FROM_IMPACT) ? 1 : 0,
-        accept, choice, final_commit, y, L);
-    return launch_result();
+    return launch_result(pvf_launch(pvf_verify_kernel, dim3(n_seq), dim3(kThreads), 0, (cudaStream_t)stream,
+                                    seg_off, row_pos, rem_rows, rem_off, v_off, draft_rows, n_drafts, route, tok,
+                                    tok_v, conf_v, commit, params->tau_high, params->budget,
+                                    (params->flags & PVF_EXCLUDE_SELF_FROM_IMPACT) ? 1 : 0, accept, choice,
+                                    final_commit, y, L));
 }
 
 }  // extern "C"

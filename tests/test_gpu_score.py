@@ -36,9 +36,12 @@ def test_config0_tiny(stress):
 
 
 @pytest.mark.parametrize("V,D,M", [(4096, 256, 1), (4096, 256, 7), (4096, 256, 128), (4096, 256, 129),
-                                   (5000, 200, 150), (1000, 64, 33), (16, 8, 3), (70000, 512, 300)])
+                                   (5000, 200, 150), (1000, 64, 33), (16, 8, 3), (70000, 512, 300),
+                                   (4096, 256, 16), (4096, 256, 17), (4096, 256, 31), (4096, 256, 32),
+                                   (5000, 200, 20), (70000, 512, 30), (100, 64, 5), (300, 72, 9), (40000, 136, 32)])
 def test_ragged_shapes(V, D, M):
-    # several row tiles, vocabulary not a multiple of 16, hidden size not a multiple of 64
+    # several row tiles, vocabulary not a multiple of 16, hidden size not a multiple of 64; up to 32 rows
+    # take the swapped-operand streaming kernel, more rows the 128-row GEMM kernel
     pos = np.arange(M)
     st = synth.build_step("ragged", 4242, V, D, min(64, V), [(pos, np.ones(M, np.uint8))], M, M,
                           dict(tau_high=0.9, budget=4), amp_max=40.0 * (256.0 / D) ** 0.5)
@@ -71,6 +74,24 @@ def test_exact_tie_goes_to_lowest_id_across_ranges():
     ctx = make_ctx(w, [10], 8)
     got = to_np(ctx.score(upload_bits(synth.f32_to_bf16_bits(h))))
     assert got["tok"][0] == 10 and got["in_plan"][0] == 1
+    ctx.close()
+
+
+@pytest.mark.parametrize("M", [1, 20, 40])
+def test_exact_ties_inside_one_range(M):
+    # equal logits at ids that one block sees on the same accumulator lane (10 and 138), in its other
+    # 128-entry slice (138), in a later tile (300) and in another block's range (60000)
+    V, D = 70000, 64
+    w = synth.make_w(11, V, D)
+    for v in (138, 300, 60000):
+        w[v] = w[10]
+    w[20000] = w[19999]
+    h = np.zeros((M, D), np.float32)
+    h[:] = synth.bf16_bits_to_f32(w[10]).astype(np.float32) * 400.0
+    h[M - 1] = synth.bf16_bits_to_f32(w[19999]).astype(np.float32) * 400.0
+    ctx = make_ctx(w, [10], 64)
+    got = to_np(ctx.score(upload_bits(synth.f32_to_bf16_bits(h))))
+    assert (got["tok"][:M - 1] == 10).all() and got["tok"][M - 1] == 19999
     ctx.close()
 
 
