@@ -9,7 +9,7 @@
 #include "pvf.h"
 
 #define PVF_MAX_BUDGET_LIMIT 64
-#define PVF_W_BOX_LEVELS 5
+#define PVF_W_BOX_SIZES 16
 
 // Device scalars at the head of the workspace.
 struct pvf_device_words {
@@ -29,7 +29,7 @@ struct pvf_ctx {
     uint32_t *plan_bitmap;  // ceil(V/32) words, bit v set iff v in P^plan
     float4 *partials;       // [rows][splits] per-range softmax states of pvf_score
     size_t partials_bytes;
-    CUtensorMap tm_w[PVF_W_BOX_LEVELS];   // W as [V][D], boxes of 16 << level rows x 64 columns, 128-byte swizzle
+    CUtensorMap tm_w[PVF_W_BOX_SIZES];   // W as [V][D], boxes of 16 * (i + 1) rows x 64 columns, 128-byte swizzle
     cudaEvent_t ev_start, ev_stop;   // optional timing hook around the GEMM kernel
     uint8_t *staging;                // optional device staging of the host-buffer entry points
     size_t staging_bytes;

@@ -64,7 +64,7 @@ constexpr int kThreads = 192;
 constexpr int kEpilogueThreads = 128;
 constexpr int kMaxStages = 16;
 constexpr int kStreamRows = 32;            // the streaming kernel handles at most this many rows
-constexpr int kWBoxLevels = PVF_W_BOX_LEVELS;           // W boxes of 16, 32, 64, 128 and 256 vocabulary entries
+constexpr int kWBoxSizes = PVF_W_BOX_SIZES;             // W boxes of 16, 32, ..., 256 vocabulary entries
 constexpr int kMaxConcurrentTiles = 64;    // cap on the wave's L2-resident H tiles
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -93,14 +93,17 @@ struct __align__(8) SharedControl {
     unsigned long long acc_full[2];        // accumulator complete
     unsigned long long acc_empty[2];       // epilogue has drained the accumulator
     unsigned long long drain;              // abort path: all issued MMAs completed
+    unsigned long long drain2;             // the same for the streaming kernel's second issuer
     uint32_t tmem_base;
     volatile int abort_flag;
 };
 static_assert(sizeof(SharedControl) <= 512, "control block");
 
-// W as [V][D] seen through boxes of 16 << level rows x 64 columns.
+// W as [V][D] seen through boxes of 16 * n rows x 64 columns, n = 1 .. 16: a vocabulary tile of any
+// whole number of granules is one TMA instruction (the producer thread is bound by the instructions
+// it issues, not by the bytes they move).
 struct WMaps {
-    CUtensorMap level[kWBoxLevels];
+    CUtensorMap size[kWBoxSizes];
 };
 
 struct ScoreArgs {
@@ -322,30 +325,17 @@ __device__ __forceinline__ void fold16(RowState &st, const uint32_t (&raw)[16], 
     }
 }
 
-// One W tile of `tun` granules starting at granule tu0, columns x .. x+63, into b_dst: the fewest
-// boxes that cover it (a full tile is one box, a ragged one the binary expansion of its size).
-#if PVF_W_EVICT_FIRST
-#define PVF_W_LOAD(dst, level_, row) tma_load_2d_hint(dst, &maps.level[level_], full, x, row, policy)
-#else
-#define PVF_W_LOAD(dst, level_, row) tma_load_2d(dst, &maps.level[level_], full, x, row)
-#endif
-template <int kUnitsPerTile>
+// One W tile of `tun` granules starting at granule tu0, columns x .. x+63, into b_dst.
 __device__ __forceinline__ void load_w_tile(uint32_t b_dst, const WMaps &maps, uint32_t full, int x, int tu0, int tun,
                                             unsigned long long policy)
 {
+#if PVF_W_EVICT_FIRST
+    tma_load_2d_hint(b_dst, &maps.size[tun - 1], full, x, tu0 * kUnit, policy);
+#else
     (void)policy;
-    constexpr int kTop = kUnitsPerTile == 16 ? 4 : (kUnitsPerTile == 8 ? 3 : 2);
-    if (tun == kUnitsPerTile) {
-        PVF_W_LOAD(b_dst, kTop, tu0 * kUnit);
-        return;
-    }
-    int u = 0;
-    if (kUnitsPerTile > 8 && (tun & 8)) { PVF_W_LOAD(b_dst + u * kUnitBytes, 3, (tu0 + u) * kUnit); u += 8; }
-    if (kUnitsPerTile > 4 && (tun & 4)) { PVF_W_LOAD(b_dst + u * kUnitBytes, 2, (tu0 + u) * kUnit); u += 4; }
-    if (tun & 2) { PVF_W_LOAD(b_dst + u * kUnitBytes, 1, (tu0 + u) * kUnit); u += 2; }
-    if (tun & 1) { PVF_W_LOAD(b_dst + u * kUnitBytes, 0, (tu0 + u) * kUnit); }
+    tma_load_2d(b_dst, &maps.size[tun - 1], full, x, tu0 * kUnit);
+#endif
 }
-#undef PVF_W_LOAD
 
 // ---------------------------------------------------------------------------------- GEMM kernel
 template <class Cfg>
@@ -389,9 +379,7 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     }
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
-#pragma unroll
-        for (int l = 0; l < kWBoxLevels; ++l)
-            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.level[l]) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.size[kWBoxSizes - 1]) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -443,7 +431,7 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
                         for (int p = 0; p < np; ++p) {
                             const int x = (kb0 + p) * kBlockK;
                             tma_load_2d(a_base + p * Cfg::kAPanelBytes, &tm_h, full, x, m_tile * kTileM);
-                            load_w_tile<kUnitsPerTile>(b_base + p * Cfg::kBPanelBytes, tm_w, full, x, tu0, tun, policy);
+                            load_w_tile(b_base + p * Cfg::kBPanelBytes, tm_w, full, x, tu0, tun, policy);
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
@@ -579,6 +567,9 @@ constexpr int kStreamWBytes = kStreamTileN * kRowBytes;             // 32 KiB
 constexpr int kStreamStageBytes = kStreamHBytes + kStreamWBytes;
 constexpr int kStreamTmemCols = 128;                                // 2 buffers x 2 slices x 32 columns
 constexpr int kStreamControlBytes = 512;
+constexpr int kStreamIssuers = 2;                                   // MMA-issuing threads (one per vocabulary slice)
+constexpr int kStreamSecondIssuerWarp = 6;
+constexpr int kStreamThreads = 224;                                 // producer, issuer, 4 epilogue warps, issuer
 constexpr int kStreamSmemBytes = kStreamStages * kStreamStageBytes + 1024 + kStreamControlBytes;
 static_assert(kStreamStages >= 2 && kStreamStages <= kMaxStages && kStreamSmemBytes <= 227 * 1024, "streaming ring");
 // the end-of-block fold reuses the tile ring: 128 lanes x 32 rows x 16 bytes
@@ -619,7 +610,7 @@ __device__ __forceinline__ void state_merge(float4 &a, const float4 b)
     a.w = __int_as_float(arg);
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kStreamThreads, 1)
 pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ WMaps tm_w, const ScoreArgs args)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -641,22 +632,21 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStreamStages; ++s) {
             mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
+            mbar_init(smem_u32(&ctl->empty[s]), kStreamIssuers);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
+            mbar_init(smem_u32(&ctl->acc_full[b]), kStreamIssuers);
             mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueThreads);
         }
         mbar_init(smem_u32(&ctl->drain), 1);
+        mbar_init(smem_u32(&ctl->drain2), 1);
         ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
-#pragma unroll
-        for (int l = 0; l < kWBoxLevels; ++l)
-            asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.level[l]) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.size[kWBoxSizes - 1]) : "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -689,7 +679,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
                     mbar_arrive_expect_tx(full, bytes);
                     armed_parity[stage] = (int)phase;
                     tma_load_2d(h_dst, &tm_h, full, step * kBlockK, 0);
-                    load_w_tile<kStreamUnitsPerTile>(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, 0ull);
+                    load_w_tile(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, 0ull);
                     if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -702,9 +692,14 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
                     }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp == 1 || warp == kStreamSecondIssuerWarp) {
+        // ------------------------------------------------------------------ MMA issuers
+        // One thread per 128-entry vocabulary slice: a single thread cannot issue the eight small MMAs
+        // of a stage as fast as the stage's bytes arrive.  Both commit every stage and every tile (a
+        // commit with nothing outstanding arrives at once), so the barrier counts never depend on
+        // how many slices a ragged tile has.
         if (lane == 0) {
+            const int sl = warp == 1 ? 0 : 1;                            // this thread's slice
             int stage = 0;
             uint32_t phase = 0;
             bool alive = true;
@@ -723,7 +718,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
                     tc_fence_after_sync();
                     const uint32_t h_addr = tiles_addr + stage * kStreamStageBytes;
                     const uint64_t h_desc = smem_desc_k_major_sw128(h_addr);
-                    for (int sl = 0; sl < n_slices; ++sl) {
+                    if (sl < n_slices) {
                         // Slice sl = rows sl*128 .. sl*128+127 of the W tile.  A ragged tile's last slice reads
                         // rows past its end: stale bytes of the same stage, on lanes the epilogue skips.
                         const uint64_t w_desc = smem_desc_k_major_sw128(h_addr + kStreamHBytes + sl * (kTileM * kRowBytes));
@@ -738,9 +733,10 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
                 if (alive) tc_commit(smem_u32(&ctl->acc_full[buf]));
             }
             if (!alive) {
-                tc_commit(smem_u32(&ctl->drain));
+                const uint32_t drain = smem_u32(sl == 0 ? &ctl->drain : &ctl->drain2);
+                tc_commit(drain);
                 const unsigned long long t0 = global_timer_ns();
-                while (!mbar_try_wait(smem_u32(&ctl->drain), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try_wait(drain, 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
             }
         }
     } else {
@@ -905,8 +901,8 @@ int make_tensor_map(CUtensorMap *map, const void *base, uint64_t rows, uint64_t 
 
 int make_w_maps(CUtensorMap *levels, const void *w_head, int vocab, int hidden)
 {
-    for (int l = 0; l < kWBoxLevels; ++l) {
-        const int rc = make_tensor_map(&levels[l], w_head, (uint64_t)vocab, (uint64_t)hidden, (uint32_t)(kUnit << l));
+    for (int l = 0; l < kWBoxSizes; ++l) {
+        const int rc = make_tensor_map(&levels[l], w_head, (uint64_t)vocab, (uint64_t)hidden, (uint32_t)(kUnit * (l + 1)));
         if (rc != PVF_OK) return rc;
     }
     return PVF_OK;
@@ -931,7 +927,7 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
     int rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)g.a_rows);
     if (rc != PVF_OK) return rc;
     WMaps maps;
-    for (int l = 0; l < kWBoxLevels; ++l) maps.level[l] = w_levels[l];
+    for (int l = 0; l < kWBoxSizes; ++l) maps.size[l] = w_levels[l];
 
     ScoreArgs a;
     a.M = M; a.V = V; a.D = D;
@@ -945,7 +941,7 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
     if (timed && cudaEventRecord(ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
     cudaError_t e;
     if (g.streaming)
-        e = pvf_launch(pvf_score_stream_kernel, dim3(g.ctas), dim3(kThreads), kStreamSmemBytes, s, tm_h, maps, a);
+        e = pvf_launch(pvf_score_stream_kernel, dim3(g.ctas), dim3(kStreamThreads), kStreamSmemBytes, s, tm_h, maps, a);
     else
         e = pvf_launch(pvf_score_gemm_kernel<GeneralCfg>, dim3(g.ctas), dim3(kThreads), GeneralCfg::kSmemBytes, s, tm_h, maps, a);
     if (e != cudaSuccess) return PVF_ERR_CUDA;
@@ -1110,7 +1106,7 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     const pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden_size, st->n_sm);
     if ((size_t)M * g.splits * sizeof(float4) > kStaticPartialsBytes) return PVF_ERR_TOO_LARGE;
 
-    CUtensorMap w_levels[kWBoxLevels];
+    CUtensorMap w_levels[kWBoxSizes];
     if ((rc = make_w_maps(w_levels, w_head, vocab, hidden_size)) != PVF_OK) return rc;
 
     cudaStream_t s = (cudaStream_t)stream;
