@@ -34,11 +34,12 @@ if ROOT not in sys.path:
 METRIC = "masked positions scored/s per fused PVF step"
 UNIT = "positions/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one GEMM launch, from the ncu captures
-# summarised under profiles/: the config-1a launch was captured as is; larger workloads scale the
-# compute-bound capture (3 passes over W, 13704 rows: 3.636 GB) by their number of passes ("waves").
-NCU_TRAFFIC_CFG1A = 1.0408e9
-NCU_TRAFFIC_PER_WAVE = 3.636e9 / 3
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the projection kernel, from
+# the ncu captures summarised under profiles/ (None = not captured since the kernel last changed).  The
+# streaming kernel's config-1a launch is captured as is; launches of the GEMM kernel scale the captured
+# per-pass traffic by their number of passes over W ("waves").
+NCU_TRAFFIC_STREAM_LAUNCH = 1.04074e9
+NCU_TRAFFIC_GEMM_PER_WAVE = 1.244e9
 
 
 def load_peaks():
@@ -296,11 +297,14 @@ def run_ours(args):
     else:
         roof = dict(bound="tensor", achieved=alg_flops / t_gemm / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
-    if args.workload == "cfg1a":
-        traffic = NCU_TRAFFIC_CFG1A
+    kernels = sorted({ctx.score_kernel_name(r) for _, _, r in ev_pairs})
+    if kernels == ["pvf_score_stream_kernel"]:
+        traffic = NCU_TRAFFIC_STREAM_LAUNCH
+    elif kernels == ["pvf_score_gemm_kernel"] and NCU_TRAFFIC_GEMM_PER_WAVE is not None:
+        traffic = NCU_TRAFFIC_GEMM_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
     else:
-        traffic = NCU_TRAFFIC_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
-    roof.update(traffic=traffic, kernel="pvf_score_gemm_kernel", launches=n_gemm, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
+        traffic = None
+    roof.update(traffic=traffic, kernel="+".join(kernels), launches=n_gemm, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
                 algorithmic_bytes_per_launch=alg_bytes / max(n_gemm, 1), peak_source=peaks["source"] +
                 (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy bandwidth)"))
 

@@ -111,6 +111,11 @@ int pvf_last_status(pvf_ctx *ctx, int32_t *status);
  */
 int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int32_t *waves, int32_t *launches);
 
+/* Name of the projection kernel pvf_score launches for M rows (for profiler filters and reports):
+ * "pvf_score_stream_kernel" up to 32 rows (vocabulary on the accumulator lanes, rows on its columns),
+ * "pvf_score_gemm_kernel" above (rows on the lanes).  NULL on an invalid argument. */
+const char *pvf_score_kernel_name(pvf_ctx *ctx, int32_t M);
+
 /*
  * Timing hook for benchmarks.  While both events (cudaEvent_t passed as void*) are non-NULL, every
  * pvf_score call records `start` immediately before and `stop` immediately after its GEMM kernel on
@@ -242,7 +247,7 @@ int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hid
  *   tok, conf, ent, in_plan   outputs as in pvf_score (ent and in_plan may be NULL)
  *
  * The call itself allocates nothing: no cudaMalloc / cudaFree, no allocating library routine; it
- * encodes three tensor maps on the host, clears one status word with cudaMemsetAsync and launches the two
+ * encodes its tensor maps on the host, clears one status word with cudaMemsetAsync and launches the two
  * scoring kernels on `stream`.  The first call on each device additionally looks up the array's device
  * address and raises the GEMM kernel's shared-memory limit (this also makes the CUDA runtime load the
  * kernels); make that first call with the device current and before any stream capture begins.

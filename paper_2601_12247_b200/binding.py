@@ -62,6 +62,7 @@ def load() -> ctypes.CDLL:
         lib.pvf_last_status.argtypes = [vp, ctypes.POINTER(i32)]; lib.pvf_last_status.restype = ctypes.c_int
         lib.pvf_set_score_events.argtypes = [vp, vp, vp]; lib.pvf_set_score_events.restype = ctypes.c_int
         lib.pvf_score_plan.argtypes = [vp, i32] + [ctypes.POINTER(i32)] * 4; lib.pvf_score_plan.restype = ctypes.c_int
+        lib.pvf_score_kernel_name.argtypes = [vp, i32]; lib.pvf_score_kernel_name.restype = ctypes.c_char_p
         lib.pvf_score.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]; lib.pvf_score.restype = ctypes.c_int
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
@@ -156,6 +157,12 @@ class Context:
         v = [ctypes.c_int32() for _ in range(4)]
         _check(self.lib.pvf_score_plan(self.handle, int(M), *[ctypes.byref(x) for x in v]), "pvf_score_plan")
         return dict(ctas=v[0].value, splits=v[1].value, waves=v[2].value, launches=v[3].value)
+
+    def score_kernel_name(self, M: int) -> str:
+        name = self.lib.pvf_score_kernel_name(self.handle, int(M))
+        if name is None:
+            raise PvfError(PVF_ERR_INVALID, "pvf_score_kernel_name")
+        return name.decode()
 
     # ------------------------------------------------------------------ host-buffer variants
     def attach_host_staging(self):

@@ -1026,6 +1026,13 @@ int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int3
     return PVF_OK;
 }
 
+const char *pvf_score_kernel_name(pvf_ctx *ctx, int32_t M)
+{
+    if (!ctx || M <= 0 || M > ctx->shape.max_rows) return nullptr;
+    const pvf_score_geometry g = pvf_score_geometry_for(M, ctx->shape.vocab, ctx->shape.hidden, ctx->n_sm);
+    return g.streaming ? "pvf_score_stream_kernel" : "pvf_score_gemm_kernel";
+}
+
 int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
               int32_t *tok, float *conf, float *ent, uint8_t *in_plan, void *stream)
 {
