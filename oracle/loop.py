@@ -8,7 +8,8 @@ block's masked positions.  One loop step = one batched forward (draft pass and v
 branches counted together).
 
 `decode(..., budget=0)` is confidence-threshold decoding (Section 2): nothing is drafted, every
-step commits the base set only.
+step commits the base set only.  `n_sparse` is the early cross-block threshold N_s (Appendix,
+"Planning-Guided Early Cross-Block Revelation", Eq. 4; 0 = strict block order).
 """
 from __future__ import annotations
 
@@ -20,25 +21,42 @@ from . import score as oscore
 from . import step as ostep
 
 
-def working_rows(y: np.ndarray, mask_id: int, block: int):
-    """Rows of the current step: for each unfinished sequence the masked positions of its first
-    block that holds a mask.  Returns seq_ids, positions (ascending per sequence), seg_off."""
+def working_set(y: np.ndarray, mask_id: int, block: int, n_sparse: int = 0):
+    """Rows of the current step with early cross-block revelation (Appendix, Eq. 4).
+
+    For each sequence: k_t is the first block that holds a mask and M_active its masked
+    positions.  The working index set B_t is M_active, widened by the whole index range of
+    block k_t + 1 when |M_active| <= N_s (``n_sparse``) and that block exists.  The scored rows
+    are the masked positions of B_t, ascending.  N_s = 0 never widens (|M_active| >= 1).
+    Returns seq_ids, positions, seg_off and the per-sequence flag ``expanded``."""
     n_seq, L = y.shape
     seq_ids, positions = [], []
     seg_off = np.zeros(n_seq + 1, dtype=np.int32)
+    expanded = np.zeros(n_seq, dtype=np.uint8)
     for b in range(n_seq):
-        masked = np.nonzero(y[b] == mask_id)[0]
-        if len(masked):
-            k = int(masked[0]) // block
-            pos = [int(i) for i in masked if k * block <= i < (k + 1) * block]
+        masked = [int(i) for i in range(L) if y[b, i] == mask_id]
+        if masked:
+            k = masked[0] // block                               # k_t (0-based)
+            m_active = [i for i in masked if k * block <= i < (k + 1) * block]
+            b_t = set(m_active)
+            if len(m_active) <= n_sparse and (k + 1) * block < L:
+                b_t |= set(range((k + 1) * block, min((k + 2) * block, L)))   # I_{k_t+1}
+                expanded[b] = 1
+            pos = [i for i in masked if i in b_t]
             seq_ids.extend([b] * len(pos))
             positions.extend(pos)
         seg_off[b + 1] = len(positions)
-    return np.asarray(seq_ids, np.int32), np.asarray(positions, np.int32), seg_off
+    return np.asarray(seq_ids, np.int32), np.asarray(positions, np.int32), seg_off, expanded
+
+
+def working_rows(y: np.ndarray, mask_id: int, block: int, n_sparse: int = 0):
+    """seq_ids, positions (ascending per sequence), seg_off of the current step's rows."""
+    seq_ids, positions, seg_off, _ = working_set(y, mask_id, block, n_sparse)
+    return seq_ids, positions, seg_off
 
 
 def decode(synth, w_bits, plan_ids, targets, seed: int, gen_len: int, block: int, params: Dict,
-           mask_id: int, max_steps: int = 100000, trace: bool = False) -> Dict:
+           mask_id: int, max_steps: int = 100000, trace: bool = False, n_sparse: int = 0) -> Dict:
     """Run Algorithm 1 until no masks remain.  ``synth`` is the input-generator module."""
     n_seq = targets.shape[0]
     K = int(params["budget"])
@@ -50,7 +68,7 @@ def decode(synth, w_bits, plan_ids, targets, seed: int, gen_len: int, block: int
     while (y == mask_id).any():
         if n_steps >= max_steps:
             raise RuntimeError("decode loop did not terminate")
-        seq_ids, positions, seg_off = working_rows(y, mask_id, block)
+        seq_ids, positions, seg_off = working_rows(y, mask_id, block, n_sparse)
         frac = (y != mask_id).sum(axis=1) / float(gen_len)
         h = synth.loop_hidden(w_bits, targets, seed, n_steps, 0, seq_ids, positions, frac)
         sc = oscore.score(w_bits, h, plan_ids)

@@ -81,3 +81,22 @@ def test_pvf_needs_no_more_forwards_than_threshold_decoding_here():
     r0 = oloop.decode(synth, w, plan, tg, SEED, L, S, dict(P, budget=0), MASK)
     assert r["steps_per_seq"].sum() <= r0["steps_per_seq"].sum()
     assert r["tokens_per_forward"] >= 1.0
+
+
+def test_early_cross_block_revelation_loop_terminates_and_never_skips_ahead():
+    # Eq. 4: with N_s > 0 the loop may fill positions of block k+1 while block k still holds masks,
+    # but never anything beyond block k+1; it still terminates and never changes a committed token.
+    w, plan, tg = setup()
+    r = oloop.decode(synth, w, plan, tg, SEED, L, S, P, MASK, trace=True, n_sparse=6)
+    assert not (r["y"] == MASK).any()
+    prev = np.full((B, L), MASK, np.int32)
+    for h in r["history"]:
+        keep = prev != MASK
+        assert np.array_equal(h["y"][keep], prev[keep])
+        for b in range(B):
+            masked = np.nonzero(prev[b] == MASK)[0]
+            if len(masked):
+                k = masked[0] // S
+                new = np.nonzero((h["y"][b] != MASK) & (prev[b] == MASK))[0]
+                assert np.all(new < (k + 2) * S)
+        prev = h["y"]
