@@ -199,6 +199,28 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
                int32_t *y, int32_t L, void *stream);
 
 /*
+ * pvf_working_set -- the rows of the next step, from the canvas (Appendix A.1, semi-autoregressive block
+ * order; Appendix "Planning-Guided Early Cross-Block Revelation", Eq. 4).
+ *   y          [n_seq][L] canvas, mask_id marks a masked position; block = S tokens per block (the last
+ *              block is shorter when S does not divide L).
+ * Per sequence: k_t = the first block that holds a mask, M_active = its masked positions; the working index
+ * set B_t is M_active, plus the whole index range of block k_t + 1 when |M_active| <= n_sparse (N_s) and
+ * that block exists.  The rows are the masked positions of B_t, ascending; n_sparse = 0 is strict block order.
+ * Outputs
+ *   seg_off   [n_seq+1]   row offsets per sequence; seg_off[n_seq] = M, the number of rows (read it back to
+ *                         size the forward pass and the pvf_score call)
+ *   row_pos   [M]         canvas position of each row          row_seq [M]  its sequence       (may be NULL)
+ *   active    [M]         1 for every row written (all of them lie in B_t)                     (may be NULL)
+ *   expanded  [n_seq]     1 where the next block was revealed                                  (may be NULL)
+ * rows_capacity = entries available in row_pos / row_seq / active; at least n_seq * min(2 * block, L), else
+ * PVF_ERR_INVALID and nothing is launched.  A finished sequence owns no rows.
+ */
+int pvf_working_set(pvf_ctx *ctx, const int32_t *y, int32_t n_seq, int32_t L, int32_t block,
+                    int32_t n_sparse, int32_t mask_id, int32_t *seg_off, int32_t *row_pos,
+                    int32_t *row_seq, uint8_t *active, uint8_t *expanded, int32_t rows_capacity,
+                    void *stream);
+
+/*
  * Host-buffer variants of the step (Algorithm 1, one decoding iteration split at the model's
  * verification forward).  Every array argument is a HOST pointer (pinned memory makes the copies
  * asynchronous); the library copies inputs into a device staging buffer, runs the device entry points

@@ -67,6 +67,8 @@ def load() -> ctypes.CDLL:
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
         lib.pvf_verify.argtypes = [vp, pp, i32, i32] + [vp] * 16 + [i32, vp]; lib.pvf_verify.restype = ctypes.c_int
+        lib.pvf_working_set.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp]
+        lib.pvf_working_set.restype = ctypes.c_int
         lib.pvf_host_staging_bytes.argtypes = [ps]; lib.pvf_host_staging_bytes.restype = sz
         lib.pvf_attach_host_staging.argtypes = [vp, vp, sz]; lib.pvf_attach_host_staging.restype = ctypes.c_int
         lib.pvf_draft_step_host.argtypes = [vp, pp, vp, i32, i32] + [vp] * 14 + [vp]; lib.pvf_draft_step_host.restype = ctypes.c_int
@@ -191,6 +193,24 @@ class Context:
         rc = self.lib.pvf_verify_step_host(self.handle, ctypes.byref(params), _ptr(hidden_v_host), Mv,
                                            hp("tok_v"), hp("conf_v"), hp("accept"), hp("choice"), hp("final_commit"), _stream())
         _check(rc, "pvf_verify_step_host")
+        return out
+
+    def working_set(self, y: torch.Tensor, block: int, n_sparse: int, mask_id: int, out=None):
+        """pvf_working_set: rows of the next step from the canvas y [n_seq][L] (int32, on the device)."""
+        assert y.is_cuda and y.dtype == torch.int32 and y.is_contiguous() and y.dim() == 2
+        n_seq, L = y.shape
+        cap = n_seq * min(2 * int(block), L)
+        if out is None:
+            dev = self.device
+            out = dict(seg_off=torch.empty(n_seq + 1, dtype=torch.int32, device=dev),
+                       row_pos=torch.empty(max(cap, 1), dtype=torch.int32, device=dev),
+                       row_seq=torch.empty(max(cap, 1), dtype=torch.int32, device=dev),
+                       active=torch.empty(max(cap, 1), dtype=torch.uint8, device=dev),
+                       expanded=torch.empty(max(n_seq, 1), dtype=torch.uint8, device=dev))
+        rc = self.lib.pvf_working_set(self.handle, _ptr(y), n_seq, L, int(block), int(n_sparse), int(mask_id),
+                                      _ptr(out["seg_off"]), _ptr(out["row_pos"]), _ptr(out.get("row_seq")),
+                                      _ptr(out.get("active")), _ptr(out.get("expanded")), out["row_pos"].shape[0], _stream())
+        _check(rc, "pvf_working_set")
         return out
 
     # ------------------------------------------------------------------ the four calls

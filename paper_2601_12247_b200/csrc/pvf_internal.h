@@ -15,7 +15,8 @@
 struct pvf_device_words {
     int32_t  status;        // PVF_OK or PVF_ERR_TIMEOUT, written by kernels
     uint32_t select_ticket; // blocks of pvf_select_drafts that have finished; reset by the last one
-    uint32_t pad[62];
+    uint32_t working_ticket; // the same for pvf_working_set
+    uint32_t pad[61];
 };
 
 struct pvf_ctx {

@@ -4,7 +4,8 @@ The transformer is replaced by the seeded generator of ``synth``: at every step 
 the scored rows are re-drawn on the host from (seed, step, sequence, position), with an amplitude that
 grows with the sequence's committed fraction, and uploaded.  Decoding is semi-autoregressive: the
 working block of a sequence is its first block that still holds a mask; the scored rows are that block's
-masked positions.  One step = draft-pass score, commit, draft selection, verification-pass score, verify;
+masked positions, widened by the next block under early cross-block revelation (``n_sparse``); the rows
+come from pvf_working_set on the device.  One step = draft-pass score, commit, draft selection, verification-pass score, verify;
 it counts as one batched forward.  ``budget = 0`` gives confidence-threshold decoding.
 
 This is a harness around the library (the hot path is the five kernels); it reports steps,
@@ -24,26 +25,12 @@ import torch
 from . import binding, synth
 
 
-def working_rows(y: np.ndarray, mask_id: int, block: int):
-    """Masked positions of each unfinished sequence's first block that holds a mask."""
-    n_seq, L = y.shape
-    masked = y == mask_id
-    has = masked.any(axis=1)
-    first = np.where(has, masked.argmax(axis=1), 0)
-    blk = first // block
-    pos_grid = np.arange(L)[None, :]
-    in_block = (pos_grid >= (blk * block)[:, None]) & (pos_grid < ((blk + 1) * block)[:, None])
-    take = masked & in_block & has[:, None]
-    seq_ids, positions = np.nonzero(take)                      # row-major: sequences, then ascending position
-    seg_off = np.concatenate([[0], np.cumsum(take.sum(axis=1))]).astype(np.int32)
-    return seq_ids.astype(np.int32), positions.astype(np.int32), seg_off
-
-
 def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: int, gen_len: int, block: int,
            params: Dict, mask_id: int, max_steps: int = 100000,
-           on_step: Optional[Callable[[int, Dict], None]] = None) -> Dict:
+           on_step: Optional[Callable[[int, Dict], None]] = None, n_sparse: int = 0) -> Dict:
     """Run the loop until no masks remain.  ``params`` holds tau_high, tau_plan_lo, tau_plan_hi, tau_ar_lo
-    and budget.  Returns y, step counts, scored rows and kernel times."""
+    and budget; ``n_sparse`` is the early cross-block threshold N_s (Eq. 4; 0 = strict block order).
+    Returns y, step counts, scored rows and kernel times."""
     dev = ctx.device
     n_seq = targets.shape[0]
     K = int(params["budget"])
@@ -53,15 +40,18 @@ def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: 
     y = np.full((n_seq, gen_len), mask_id, dtype=np.int32)
     steps_per_seq = np.zeros(n_seq, dtype=np.int32)
     scored_rows, n_steps, kernel_ms = 0, 0, 0.0
-    to_dev = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(dev)
     while (y == mask_id).any():
         if n_steps >= max_steps:
             raise RuntimeError("decode loop did not terminate")
-        seq_ids, positions, seg_off = working_rows(y, mask_id, block)
+        ws = ctx.working_set(y_dev, block, n_sparse, mask_id)          # rows of this step, built on the device
+        seg_off = ws["seg_off"].cpu().numpy()
+        n_rows = int(seg_off[-1])
+        positions = ws["row_pos"][:n_rows].cpu().numpy()
+        seq_ids = ws["row_seq"][:n_rows].cpu().numpy()
         frac = (y != mask_id).sum(axis=1) / float(gen_len)
         h_bits = synth.loop_hidden(w_bits, targets, seed, n_steps, 0, seq_ids, positions, frac)
         h = binding.bf16_from_bits(h_bits, dev)
-        seg, pos = to_dev(seg_off, np.int32), to_dev(positions, np.int32)
+        seg, pos = ws["seg_off"], ws["row_pos"][:n_rows]
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         e[0].record()
         sc = ctx.score(h)
@@ -114,6 +104,7 @@ def main():
     ap.add_argument("--budget", type=int, default=4)
     ap.add_argument("--n-plan", type=int, default=2048)
     ap.add_argument("--q-plan", type=float, default=0.0, help="fraction of targets drawn from the planning ids")
+    ap.add_argument("--n-sparse", type=int, default=0, help="early cross-block threshold N_s (Eq. 4)")
     ap.add_argument("--seed", type=int, default=1004)
     args = ap.parse_args()
     dev = torch.device("cuda:0")
@@ -125,12 +116,13 @@ def main():
     p = dict(tau_high=0.9, budget=args.budget, **synth.DEFAULT_BAND)
     out = {}
     for name, budget in (("pvf", args.budget), ("threshold_only", 0)):
-        r = decode(ctx, w_bits, targets, args.seed, args.gen_len, args.block, dict(p, budget=budget), args.vocab - 128)
+        r = decode(ctx, w_bits, targets, args.seed, args.gen_len, args.block, dict(p, budget=budget), args.vocab - 128,
+                   n_sparse=args.n_sparse)
         out[name] = dict(steps=r["steps"], mean_steps_per_sequence=float(r["steps_per_seq"].mean()),
                          tokens_per_forward=r["tokens_per_forward"], scored_rows=r["scored_rows"],
                          kernel_ms_per_step=r["kernel_ms_per_step"], status=r["status"])
     out["config"] = dict(vocab=args.vocab, hidden=args.hidden, n_seq=args.n_seq, gen_len=args.gen_len, block=args.block,
-                         budget=args.budget, q_plan=args.q_plan, data="synthetic")
+                         budget=args.budget, q_plan=args.q_plan, n_sparse=args.n_sparse, data="synthetic")
     print(json.dumps(out))
 
 

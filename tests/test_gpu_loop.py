@@ -9,18 +9,6 @@ from paper_2601_12247_b200 import binding, decode_loop, synth
 from gpu_util import FRAGILE, NEAR_TIE, check_score, dev, make_ctx, to_np
 
 
-def test_working_rows_matches_oracle_rule():
-    rng = np.random.default_rng(0)
-    for _ in range(20):
-        y = rng.integers(0, 50, (5, 64)).astype(np.int32)
-        y[rng.random((5, 64)) < 0.5] = 99
-        y[0] = 3                                             # a finished sequence
-        a = decode_loop.working_rows(y, 99, 16)
-        b = oloop.working_rows(y, 99, 16)
-        for u, v in zip(a, b):
-            assert np.array_equal(u, v)
-
-
 def fragile_step(h, p):
     """True if the oracle's step holds a row whose decision could legitimately flip on the GPU."""
     def bad(sc, taus):
@@ -32,18 +20,18 @@ def fragile_step(h, p):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("budget,q_plan", [(4, 0.5), (0, 0.0), (3, 0.0)])
-def test_loop_tiny_shape_state_by_state(budget, q_plan):
+@pytest.mark.parametrize("budget,q_plan,n_sparse", [(4, 0.5, 0), (0, 0.0, 0), (3, 0.0, 0), (4, 0.5, 5), (0, 0.0, 8)])
+def test_loop_tiny_shape_state_by_state(budget, q_plan, n_sparse):
     V, D, B, L, S, seed = 4096, 256, 4, 64, 32, 1004
     w = synth.make_w(seed, V, D)
     plan = synth.make_plan_ids(seed, V, 256)
     tg = synth.loop_targets(seed, V, B, L, plan, q_plan, avoid=V - 1)
     p = dict(tau_high=0.9, budget=budget, **synth.DEFAULT_BAND)
     mask = V - 1
-    want = oloop.decode(synth, w, plan, tg, seed, L, S, p, mask, trace=True)
-    ctx = make_ctx(w, plan, B * S * (2 + budget), B, max(budget, 1))
+    want = oloop.decode(synth, w, plan, tg, seed, L, S, p, mask, trace=True, n_sparse=n_sparse)
+    ctx = make_ctx(w, plan, B * 2 * S * (2 + budget), B, max(budget, 1))
     trace = []
-    got = decode_loop.decode(ctx, w, tg, seed, L, S, p, mask, on_step=lambda s, d: trace.append(d))
+    got = decode_loop.decode(ctx, w, tg, seed, L, S, p, mask, on_step=lambda s, d: trace.append(d), n_sparse=n_sparse)
     assert got["status"] == 0
     n_same = 0
     for s, (g, o) in enumerate(zip(trace, want["history"])):
