@@ -8,7 +8,10 @@ with the CUDA library and never imports it.
   score.py   logits -> (top-1 token, confidence, entropy, top-2 gap, planning eligibility);
              thin ctypes wrapper around pvf_oracle_score.c
   step.py    base commit, planning / AR draft proposal, impact-set verification, branch choice
-  loop.py    Algorithm 1 on synthetic hidden states, and the threshold-only loop
+  loop.py    Algorithm 1 on synthetic hidden states, the threshold-only loop, and the working
+             set with early cross-block revelation (Eq. 4)
+  calib.py   verified information gain, per-token calibration statistics and the filtering
+             rule that builds the planning-token vocabulary
 
 Pins (tests/test_oracle_*.py): closed forms (uniform row, identity weights), invariances,
 scipy's fp64 log_softmax on tiny shapes, brute-force argmax / top-k, a streaming recurrence

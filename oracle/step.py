@@ -72,13 +72,19 @@ def commit(conf, tok, seg_off, row_pos, active, tau_high: float, force_progress:
 
 
 def select_drafts(conf, tok, in_plan, commit_mask, seg_off, row_pos, active, tau_plan_lo: float,
-                  tau_plan_hi: float, tau_ar_lo: float, budget: int) -> Dict[str, np.ndarray]:
+                  tau_plan_hi: float, tau_ar_lo: float, budget: int, any_token: bool = False,
+                  ar_fallback: bool = True) -> Dict[str, np.ndarray]:
     """Draft proposal of one step (Sections 4.1 and 4.3).
 
     Planning candidates  P_t^plan = {i in M_t \\ S_base : y^_i in P^plan, tau_l <= p_i < tau_u};
     the K_t = min(K, |P_t^plan|) most confident are the drafts, in rank order (route 1).
     If P_t^plan is empty the AR fallback proposes the leftmost <= K positions of M_t \\ S_base
     with p_i >= tau_AR^l, in position order (route 2).  Route 0: nothing to propose.
+
+    ``any_token`` drops the planning-vocabulary condition and ``ar_fallback=False`` the second route:
+    together they give the candidate set of the offline calibration, C_t^cal = {i in M_t \\ S_base :
+    tau_cal^l <= p_i < tau_cal^u} (Appendix, planning-token set construction), capped at the K most
+    confident.
 
     Also returns the remaining rows R_b = active, not base-committed rows of each sequence
     (rem_rows / rem_off) and the row offsets v_off of the verification pass, whose rows are laid
@@ -100,13 +106,13 @@ def select_drafts(conf, tok, in_plan, commit_mask, seg_off, row_pos, active, tau
         rem = [m for m in range(int(seg_off[b]), int(seg_off[b + 1])) if act[m] and not commit_mask[m]]
         rem_rows.extend(rem)
         rem_off[b + 1] = rem_off[b] + len(rem)
-        plan = [m for m in rem if in_plan[m] and lo <= conf[m] < hi]
+        plan = [m for m in rem if (any_token or in_plan[m]) and lo <= conf[m] < hi]
         chosen = []
         if K > 0 and plan:
             order = sorted(plan, key=lambda m: (-conf[m], int(row_pos[m])))
             chosen = order[:K]
             route[b] = ROUTE_PLAN
-        elif K > 0:
+        elif K > 0 and ar_fallback:
             chosen = [m for m in rem if conf[m] >= ar][:K]
             route[b] = ROUTE_AR if chosen else ROUTE_NONE
         n_drafts[b] = len(chosen)
