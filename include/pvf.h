@@ -65,6 +65,11 @@ typedef struct {
 #define PVF_FORCE_PROGRESS            1u  /* a sequence with active rows but an empty base set commits its
                                              single most confident active row (lowest position on ties) */
 #define PVF_EXCLUDE_SELF_FROM_IMPACT  2u  /* leave draft j's own position out of the impact set of branch j */
+#define PVF_SELECT_ANY_TOKEN          4u  /* pvf_select_drafts: drop the "top-1 token in P^plan" condition */
+#define PVF_NO_AR_FALLBACK            8u  /* pvf_select_drafts: no AR route when there is no planning candidate.
+                                             Both together, with the band set to the calibration band, select the
+                                             calibration candidates C_t^cal (Appendix, planning-token set
+                                             construction), at most `budget` per sequence, most confident first */
 
 /* Thresholds of the step.  Names follow the paper: tau_high (Section 2), the planning band
  * [tau_plan_lo, tau_plan_hi) (Section 4.1), tau_ar_lo (Section 4.3), budget = K drafts per sequence. */
@@ -155,11 +160,12 @@ int pvf_commit(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
  * pvf_select_drafts -- draft proposal (Section 4.1 planning candidates and TopK; Section 4.3 AR
  * candidate construction; Algorithm 1, route switch).
  * Per sequence b, with R_b = its rows that are active and not in `commit`, in position order:
- *   planning candidates = rows of R_b with in_plan != 0 and tau_plan_lo <= conf < tau_plan_hi;
+ *   planning candidates = rows of R_b with in_plan != 0 and tau_plan_lo <= conf < tau_plan_hi
+ *     (in_plan is ignored, and may be NULL, under PVF_SELECT_ANY_TOKEN);
  *   if there are any (and budget > 0): the K_t = min(budget, count) most confident, ties to the lower
  *     position, written in rank order; route = 1.
  *   otherwise: the first <= budget rows of R_b with conf >= tau_ar_lo, in position order; route = 2,
- *     or route = 0 when there is none.
+ *     or route = 0 when there is none (always route = 0 under PVF_NO_AR_FALLBACK).
  * Outputs
  *   draft_rows [n_seq][budget]  row indices, -1 padded         n_drafts [n_seq]
  *   route      [n_seq]          0 none, 1 planning, 2 AR
@@ -197,6 +203,53 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
                const int32_t *tok, const int32_t *tok_v, const float *conf_v, const uint8_t *commit,
                uint8_t *accept, int32_t *choice, uint8_t *final_commit,
                int32_t *y, int32_t L, void *stream);
+
+/*
+ * Offline construction of the planning-token vocabulary (Section 3, "Verified information gain" and
+ * "Planning-token vocabulary"; Appendix, "Planning Token Set Construction").
+ *
+ * A calibration step is a decode step on the calibration data with candidates chosen by
+ * pvf_select_drafts under PVF_SELECT_ANY_TOKEN | PVF_NO_AR_FALLBACK and the band [tau_cal_lo, tau_cal_hi):
+ * pvf_score (with entropies) on the verification pass, pvf_verify for the acceptance A_j, then
+ *
+ * pvf_calib_accumulate -- one event per candidate j of every sequence on the planning route, for the
+ * token v = tok[draft row j]:
+ *     dH_j  = mean over the remaining rows r != draft j of  ent_v[base][r] - ent_v[j][r]   (0 if there is none)
+ *     VIG_j = accept[b][j] * dH_j
+ *     n_v[v] += 1;   m_v[v] += (S_impact non-empty);   sum_a[v] += accept[b][j];
+ *     sum_vig_q32[v] += round(VIG_j * 2^32)      (integer sums: independent of the order of accumulation)
+ *   conf_v, ent_v   pvf_score outputs of the verification pass, rows as in pvf_verify
+ *   accept          pvf_verify's output for the same step
+ *   n_v, m_v, sum_a [vocab] int32 and sum_vig_q32 [vocab] int64: caller-owned, zeroed by the caller before the
+ *                   first step, accumulated across steps
+ *   vig_out         [n_seq][budget] VIG_j of this step (0 beyond n_drafts), or NULL
+ *
+ * pvf_calib_filter -- the filtering rule: bit v of plan_bitmap (ceil(vocab/32) words, fully overwritten) is set
+ * iff n_v >= n_min, m_v >= m_min, sum_a/m_v >= rho_ver (0 when m_v = 0) and (sum_vig_q32 / 2^32)/n_v >= gamma_vig;
+ * *n_plan (may be NULL) receives the number of kept tokens.
+ *
+ * pvf_set_plan_bitmap -- makes such a device bitmap the context's planning vocabulary P^plan (device-to-device
+ * copy on `stream`).
+ *
+ * pvf_default_calib_params: the paper's printed calibration band [0.15, 0.25) and thresholds n_min = 50,
+ * m_min = 20, rho_ver = 0.9, gamma_vig = 0.03.
+ */
+typedef struct {
+    float   tau_cal_lo, tau_cal_hi;
+    int32_t n_min, m_min;
+    float   rho_ver, gamma_vig;
+} pvf_calib_params;
+void pvf_default_calib_params(pvf_calib_params *out);
+int pvf_calib_accumulate(pvf_ctx *ctx, const pvf_params *params, int32_t n_seq,
+                         const int32_t *rem_rows, const int32_t *rem_off, const int32_t *v_off,
+                         const int32_t *draft_rows, const int32_t *n_drafts, const uint8_t *route,
+                         const int32_t *tok, const float *conf_v, const float *ent_v, const uint8_t *accept,
+                         int32_t *n_v, int32_t *m_v, int32_t *sum_a, int64_t *sum_vig_q32, double *vig_out,
+                         void *stream);
+int pvf_calib_filter(pvf_ctx *ctx, const pvf_calib_params *cal, const int32_t *n_v, const int32_t *m_v,
+                     const int32_t *sum_a, const int64_t *sum_vig_q32, uint32_t *plan_bitmap, int32_t *n_plan,
+                     void *stream);
+int pvf_set_plan_bitmap(pvf_ctx *ctx, const uint32_t *plan_bitmap, void *stream);
 
 /*
  * pvf_working_set -- the rows of the next step, from the canvas (Appendix A.1, semi-autoregressive block

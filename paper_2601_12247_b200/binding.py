@@ -22,6 +22,8 @@ PVF_ERR_TOO_LARGE = -7
 PVF_STATIC_MAX_ROWS = 1024
 PVF_FORCE_PROGRESS = 1
 PVF_EXCLUDE_SELF_FROM_IMPACT = 2
+PVF_SELECT_ANY_TOKEN = 4
+PVF_NO_AR_FALLBACK = 8
 
 
 class pvf_shape(ctypes.Structure):
@@ -32,6 +34,11 @@ class pvf_shape(ctypes.Structure):
 class pvf_params(ctypes.Structure):
     _fields_ = [("tau_high", ctypes.c_float), ("tau_plan_lo", ctypes.c_float), ("tau_plan_hi", ctypes.c_float),
                 ("tau_ar_lo", ctypes.c_float), ("budget", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class pvf_calib_params(ctypes.Structure):
+    _fields_ = [("tau_cal_lo", ctypes.c_float), ("tau_cal_hi", ctypes.c_float), ("n_min", ctypes.c_int32),
+                ("m_min", ctypes.c_int32), ("rho_ver", ctypes.c_float), ("gamma_vig", ctypes.c_float)]
 
 
 class PvfError(RuntimeError):
@@ -67,6 +74,11 @@ def load() -> ctypes.CDLL:
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
         lib.pvf_verify.argtypes = [vp, pp, i32, i32] + [vp] * 16 + [i32, vp]; lib.pvf_verify.restype = ctypes.c_int
+        pc = ctypes.POINTER(pvf_calib_params)
+        lib.pvf_default_calib_params.argtypes = [pc]; lib.pvf_default_calib_params.restype = None
+        lib.pvf_calib_accumulate.argtypes = [vp, pp, i32] + [vp] * 15 + [vp]; lib.pvf_calib_accumulate.restype = ctypes.c_int
+        lib.pvf_calib_filter.argtypes = [vp, pc] + [vp] * 6 + [vp]; lib.pvf_calib_filter.restype = ctypes.c_int
+        lib.pvf_set_plan_bitmap.argtypes = [vp, vp, vp]; lib.pvf_set_plan_bitmap.restype = ctypes.c_int
         lib.pvf_working_set.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp]
         lib.pvf_working_set.restype = ctypes.c_int
         lib.pvf_host_staging_bytes.argtypes = [ps]; lib.pvf_host_staging_bytes.restype = sz
@@ -87,6 +99,12 @@ def default_params() -> pvf_params:
     p = pvf_params()
     load().pvf_default_params(ctypes.byref(p))
     return p
+
+
+def default_calib_params() -> pvf_calib_params:
+    c = pvf_calib_params()
+    load().pvf_default_calib_params(ctypes.byref(c))
+    return c
 
 
 def make_params(tau_high: float, tau_plan_lo: float, tau_plan_hi: float, tau_ar_lo: float, budget: int,
@@ -194,6 +212,36 @@ class Context:
                                            hp("tok_v"), hp("conf_v"), hp("accept"), hp("choice"), hp("final_commit"), _stream())
         _check(rc, "pvf_verify_step_host")
         return out
+
+    # ------------------------------------------------------------------ planning-vocabulary calibration
+    def new_calib_stats(self) -> Dict[str, torch.Tensor]:
+        """Zeroed per-token statistics (n_v, m_v, sum_a int32; sum_vig_q32 int64) on the context's device."""
+        V = self.shape.vocab
+        z = lambda dt: torch.zeros(V, dtype=dt, device=self.device)
+        return dict(n_v=z(torch.int32), m_v=z(torch.int32), sum_a=z(torch.int32), sum_vig_q32=z(torch.int64))
+
+    def calib_accumulate(self, params: pvf_params, sel: Dict[str, torch.Tensor], tok, conf_v, ent_v, accept,
+                         stats: Dict[str, torch.Tensor], vig_out: Optional[torch.Tensor] = None):
+        n_seq = sel["n_drafts"].shape[0]
+        rc = self.lib.pvf_calib_accumulate(self.handle, ctypes.byref(params), n_seq, _ptr(sel["rem_rows"]),
+                                           _ptr(sel["rem_off"]), _ptr(sel["v_off"]), _ptr(sel["draft_rows"]),
+                                           _ptr(sel["n_drafts"]), _ptr(sel["route"]), _ptr(tok), _ptr(conf_v), _ptr(ent_v),
+                                           _ptr(accept), _ptr(stats["n_v"]), _ptr(stats["m_v"]), _ptr(stats["sum_a"]),
+                                           _ptr(stats["sum_vig_q32"]), _ptr(vig_out), _stream())
+        _check(rc, "pvf_calib_accumulate")
+
+    def calib_filter(self, cal: pvf_calib_params, stats: Dict[str, torch.Tensor]):
+        """Returns (bitmap int32 tensor of ceil(V/32) words, n_plan int32 tensor of one element)."""
+        words = (self.shape.vocab + 31) // 32
+        bitmap = torch.empty(words, dtype=torch.int32, device=self.device)
+        n_plan = torch.empty(1, dtype=torch.int32, device=self.device)
+        rc = self.lib.pvf_calib_filter(self.handle, ctypes.byref(cal), _ptr(stats["n_v"]), _ptr(stats["m_v"]),
+                                       _ptr(stats["sum_a"]), _ptr(stats["sum_vig_q32"]), _ptr(bitmap), _ptr(n_plan), _stream())
+        _check(rc, "pvf_calib_filter")
+        return bitmap, n_plan
+
+    def set_plan_bitmap(self, bitmap: torch.Tensor):
+        _check(self.lib.pvf_set_plan_bitmap(self.handle, _ptr(bitmap), _stream()), "pvf_set_plan_bitmap")
 
     def working_set(self, y: torch.Tensor, block: int, n_sparse: int, mask_id: int, out=None):
         """pvf_working_set: rows of the next step from the canvas y [n_seq][L] (int32, on the device)."""

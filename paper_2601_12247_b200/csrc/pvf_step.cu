@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(kThreads)
 pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t *__restrict__ active,
                   const float *__restrict__ conf, const uint8_t *__restrict__ in_plan,
                   const uint8_t *__restrict__ commit, float tau_lo, float tau_hi, float tau_ar, int K,
-                  int32_t *__restrict__ draft_rows, int32_t *__restrict__ n_drafts,
+                  int any_token, int ar_fallback, int32_t *__restrict__ draft_rows, int32_t *__restrict__ n_drafts,
                   uint8_t *__restrict__ route, int32_t *__restrict__ rem_rows,
                   int32_t *__restrict__ rem_off, int32_t *__restrict__ v_off, unsigned *ticket)
 {
@@ -138,7 +138,7 @@ pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t 
         if (m < r1) {
             rem = (active ? active[m] != 0 : true) && !commit[m];
             const float p = conf[m];
-            plan = rem && in_plan[m] && p >= tau_lo && p < tau_hi;  // P_t^plan
+            plan = rem && (any_token || in_plan[m]) && p >= tau_lo && p < tau_hi;  // P_t^plan
         }
         int chunk_total;
         const int rank = block_rank(rem, s_int, &chunk_total);
@@ -158,7 +158,7 @@ pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t 
             unsigned long long best = 0;
             for (int m = r0 + threadIdx.x; m < r1; m += kThreads) {
                 const float p = conf[m];
-                const bool plan = (active ? active[m] != 0 : true) && !commit[m] && in_plan[m] &&
+                const bool plan = (active ? active[m] != 0 : true) && !commit[m] && (any_token || in_plan[m]) &&
                                   p >= tau_lo && p < tau_hi;
                 if (plan) {
                     const unsigned long long k = cand_key(p, m - r0);
@@ -169,7 +169,7 @@ pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t 
             if (threadIdx.x == 0)
                 draft_rows[(size_t)b * K + j] = r0 + (int)(0xffffffffu - (unsigned)(last & 0xffffffffull));
         }
-    } else if (K > 0) {
+    } else if (K > 0 && ar_fallback) {
         // AR fallback: leftmost rows of R_b with p >= tau_AR^l, at most K of them.
         for (int c0 = r0; c0 < r1 && kt < K; c0 += kThreads) {
             const int m = c0 + threadIdx.x;
@@ -373,12 +373,14 @@ int pvf_select_drafts(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t
     (void)row_pos; (void)tok;
     if (!params_ok(ctx, params, M, n_seq)) return PVF_ERR_INVALID;
     if (n_seq == 0) return M == 0 ? PVF_OK : PVF_ERR_INVALID;
-    if (!seg_off || !conf || !in_plan || !commit || !n_drafts || !route || !rem_off || !v_off ||
+    const int any_token = (params->flags & PVF_SELECT_ANY_TOKEN) ? 1 : 0;
+    if (!seg_off || !conf || (!in_plan && !any_token) || !commit || !n_drafts || !route || !rem_off || !v_off ||
         (params->budget > 0 && !draft_rows) || (M > 0 && !rem_rows))
         return PVF_ERR_INVALID;
     return launch_result(pvf_launch(pvf_select_kernel, dim3(n_seq), dim3(kThreads), 0, (cudaStream_t)stream,
                                     n_seq, seg_off, active, conf, in_plan, commit, params->tau_plan_lo,
-                                    params->tau_plan_hi, params->tau_ar_lo, params->budget, draft_rows, n_drafts,
+                                    params->tau_plan_hi, params->tau_ar_lo, params->budget, any_token,
+                                    (params->flags & PVF_NO_AR_FALLBACK) ? 0 : 1, draft_rows, n_drafts,
                                     route, rem_rows, rem_off, v_off, &ctx->words->select_ticket));
 }
 

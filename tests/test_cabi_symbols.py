@@ -33,6 +33,10 @@ def test_defaults_are_the_papers_printed_values():
     assert p.tau_high == f32(golden["tau_high"]) and p.budget == int(golden["budget_K"])
     assert p.tau_plan_lo == f32(golden["tau_plan_lo"]) and p.tau_plan_hi == f32(golden["tau_plan_hi"])
     assert p.tau_ar_lo == f32(golden["tau_ar_lo"]) and p.flags == 0
+    c = binding.default_calib_params()
+    assert c.tau_cal_lo == f32(golden["tau_cal_lo"]) and c.tau_cal_hi == f32(golden["tau_cal_hi"])
+    assert c.n_min == int(golden["n_min"]) and c.m_min == int(golden["m_min"])
+    assert c.rho_ver == f32(golden["rho_ver"]) and c.gamma_vig == f32(golden["gamma_vig"])
     from paper_2601_12247_b200 import synth
     assert synth.DEFAULT_BAND == dict(tau_plan_lo=golden["tau_plan_lo"], tau_plan_hi=golden["tau_plan_hi"],
                                       tau_ar_lo=golden["tau_ar_lo"])
