@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the fused PVF step on one node.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1a|cfg1b|cfg2|cfg3|cfg3s]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1a|cfg1b|cfg2|cfg3|cfg3s|dream1a|dream1b]
 
 A step is one pass of the whole hot path over one synthetic batch, through the C interface:
     pvf_score(H) -> pvf_commit -> pvf_select_drafts -> pvf_score(Hv, verification pass) -> pvf_verify
@@ -53,6 +53,10 @@ def load_peaks():
 
 
 def make_workload(name: str, synth, seed_w: int = 1001):
+    if name.startswith("dream"):
+        # the second backbone's LM-head shape, same step as config 1
+        w_bits = synth.make_w(seed_w, synth.DREAM_VOCAB, synth.DREAM_HIDDEN)
+        return synth.config1(name[-1], w_bits=w_bits, vocab=synth.DREAM_VOCAB, hidden=synth.DREAM_HIDDEN)
     w_bits = synth.make_w(seed_w, synth.LLADA_VOCAB, synth.LLADA_HIDDEN)
     if name == "cfg1a":
         st = synth.config1("a", w_bits=w_bits)
@@ -387,7 +391,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg3", "cfg3s"])
+    ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg3", "cfg3s", "dream1a", "dream1b"])
     ap.add_argument("--cpu-rows", type=int, default=256, help="rows per pass the CPU baseline scores")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

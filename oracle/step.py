@@ -214,3 +214,45 @@ def c_total_margins(rem_rows, rem_off, v_off, draft_rows, n_drafts, route, conf_
         for a, c in zip(cs, cs[1:]):
             out[b] = min(out[b], c - a)
     return out
+
+
+def explore_commit(conf, tok, in_plan, commit_mask, seg_off, row_pos, active, tau_lo: float, tau_hi: float,
+                   u, planning: bool, y: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """Exploration variants of the appendix ("Planning tokens beyond high-confidence decoding"): after the
+    high-confidence commits, commit exactly one more token per sequence from the closed confidence bin
+    [tau_lo, tau_hi].
+
+    Eligible rows: active, not base-committed, tau_lo <= p <= tau_hi.  "Random" draws one of them
+    uniformly; "Planning" draws uniformly from the eligible rows whose top-1 token is in P^plan and falls
+    back to the Random rule when there is none.  The uniform draw is an input: u[b] in [0, 1) selects the
+    floor(u * n)-th of the n rows of the chosen set in position order (product taken in fp32, the precision
+    of the interface).  Returns the updated commit mask and explore_row[n_seq] (-1: bin empty).
+    """
+    conf = np.asarray(conf, dtype=np.float64)
+    M = len(conf)
+    n_seq = len(seg_off) - 1
+    act = np.ones(M, np.uint8) if active is None else np.asarray(active)
+    lo, hi = f32(tau_lo), f32(tau_hi)
+    out = np.array(commit_mask, dtype=np.uint8, copy=True)
+    explore_row = np.full(n_seq, -1, dtype=np.int32)
+    for b in range(n_seq):
+        rows = range(int(seg_off[b]), int(seg_off[b + 1]))
+        eligible = [m for m in rows if act[m] and not commit_mask[m] and lo <= conf[m] <= hi]
+        pool = eligible
+        if planning:
+            plan = [m for m in eligible if in_plan[m]]
+            if plan:
+                pool = plan
+        if pool:
+            n = len(pool)
+            idx = min(int(np.float32(u[b]) * np.float32(n)), n - 1)
+            explore_row[b] = pool[idx]
+            out[pool[idx]] = 1
+    res = dict(commit=out, explore_row=explore_row)
+    if y is not None:
+        y2 = np.array(y, copy=True)
+        for b in range(n_seq):
+            if explore_row[b] >= 0:
+                y2[b, int(row_pos[explore_row[b]])] = int(tok[explore_row[b]])
+        res["y"] = y2
+    return res

@@ -44,6 +44,11 @@ TAG_PLAN_PICK = 14
 
 LLADA_VOCAB = 126464
 LLADA_HIDDEN = 4096
+# Second backbone of the paper's experiments (Dream-7B-Instruct).  The paper states neither number; these
+# are the vocabulary and hidden size of the public Qwen2.5-7B family that model is built on, taken as a
+# second LM-head shape (hidden size not a multiple of 256, vocabulary not a multiple of the 148 blocks).
+DREAM_VOCAB = 152064
+DREAM_HIDDEN = 3584
 
 
 def _rng(seed: int, tag: int, i0: int = 0, i1: int = 0, i2: int = 0) -> np.random.Generator:

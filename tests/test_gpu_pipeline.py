@@ -194,6 +194,19 @@ def test_config2_sampled_rows_and_decisions_on_gpu_scores(llada):
         check_score(gscv, oscore.score(w_bits, v.hv_bits[rows], plan), st.vocab, plan, rows=rows)
 
 
+def test_second_model_shape_sampled():
+    # Dream-7B-like LM head: 56 k-panels, 9504 vocabulary granules (64.2 per block): both kernels
+    V, D = synth.DREAM_VOCAB, synth.DREAM_HIDDEN
+    w_bits = synth.make_w(1005, V, D)
+    plan = synth.make_plan_ids(1005, V, 2048)
+    ctx = make_ctx(w_bits, plan, 512, 8, 8)
+    for variant, sample in (("a", np.array([0, 1, 15, 16, 30, 31])), ("b", np.array([0, 127, 128, 129, 255]))):
+        st = synth.config1(variant, stress=True, w_bits=w_bits, vocab=V, hidden=D)
+        assert ctx.score_kernel_name(st.n_rows) == ("pvf_score_stream_kernel" if variant == "a" else "pvf_score_gemm_kernel")
+        sampled_parity(ctx, st, w_bits, plan, sample)
+    ctx.close()
+
+
 def test_config3_large_batch_sampled(llada):
     w_bits, plan, ctx = llada
     st = synth.config3(w_bits=w_bits)
