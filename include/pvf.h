@@ -205,6 +205,28 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
                int32_t *y, int32_t L, void *stream);
 
 /*
+ * pvf_explore_commit -- the exploration variants of the appendix ("Planning tokens beyond high-confidence
+ * decoding", the Random / Planning ablation): after pvf_commit, every sequence commits exactly one more token
+ * from the CLOSED confidence bin [tau_plan_lo, tau_plan_hi] (no verification pass).
+ *   eligible rows: active, not in `commit`, tau_plan_lo <= conf <= tau_plan_hi
+ *   PVF_EXPLORE_RANDOM    one eligible row, drawn uniformly
+ *   PVF_EXPLORE_PLANNING  one eligible row whose top-1 token is in P^plan (in_plan != 0), drawn uniformly;
+ *                         the Random rule when there is none
+ *   u [n_seq]             the draws: u[b] in [0, 1) picks row floor(u[b] * n) of the n rows of the chosen set in
+ *                         position order (fp32 product, clamped to n - 1); the caller owns the random numbers
+ * commit is updated in place (the chosen row set to 1), explore_row[b] receives the row or -1 when the bin is
+ * empty, y as in pvf_commit.  The Static baseline of the paper's tables (one most confident token per step)
+ * is pvf_commit with tau_high above 1 and PVF_FORCE_PROGRESS.
+ */
+#define PVF_EXPLORE_RANDOM   0
+#define PVF_EXPLORE_PLANNING 1
+int pvf_explore_commit(pvf_ctx *ctx, const pvf_params *params, int32_t mode, int32_t M, int32_t n_seq,
+                       const int32_t *seg_off, const int32_t *row_pos, const uint8_t *active,
+                       const int32_t *tok, const float *conf, const uint8_t *in_plan,
+                       const float *u, uint8_t *commit, int32_t *explore_row, int32_t *y, int32_t L,
+                       void *stream);
+
+/*
  * Offline construction of the planning-token vocabulary (Section 3, "Verified information gain" and
  * "Planning-token vocabulary"; Appendix, "Planning Token Set Construction").
  *

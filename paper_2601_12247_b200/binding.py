@@ -22,6 +22,7 @@ PVF_ERR_TOO_LARGE = -7
 PVF_STATIC_MAX_ROWS = 1024
 PVF_FORCE_PROGRESS = 1
 PVF_EXCLUDE_SELF_FROM_IMPACT = 2
+PVF_EXPLORE_RANDOM, PVF_EXPLORE_PLANNING = 0, 1
 PVF_SELECT_ANY_TOKEN = 4
 PVF_NO_AR_FALLBACK = 8
 
@@ -74,6 +75,8 @@ def load() -> ctypes.CDLL:
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
         lib.pvf_verify.argtypes = [vp, pp, i32, i32] + [vp] * 16 + [i32, vp]; lib.pvf_verify.restype = ctypes.c_int
+        lib.pvf_explore_commit.argtypes = [vp, pp, i32, i32, i32] + [vp] * 10 + [i32, vp]
+        lib.pvf_explore_commit.restype = ctypes.c_int
         pc = ctypes.POINTER(pvf_calib_params)
         lib.pvf_default_calib_params.argtypes = [pc]; lib.pvf_default_calib_params.restype = None
         lib.pvf_calib_accumulate.argtypes = [vp, pp, i32] + [vp] * 15 + [vp]; lib.pvf_calib_accumulate.restype = ctypes.c_int
@@ -212,6 +215,17 @@ class Context:
                                            hp("tok_v"), hp("conf_v"), hp("accept"), hp("choice"), hp("final_commit"), _stream())
         _check(rc, "pvf_verify_step_host")
         return out
+
+    def explore_commit(self, params: pvf_params, mode: int, seg_off, row_pos, active, tok, conf, in_plan, u, commit, y=None):
+        """pvf_explore_commit: updates ``commit`` in place; returns explore_row [n_seq]."""
+        M, n_seq = conf.shape[0], seg_off.shape[0] - 1
+        explore_row = torch.empty(max(n_seq, 1), dtype=torch.int32, device=self.device)
+        L = 0 if y is None else y.shape[1]
+        rc = self.lib.pvf_explore_commit(self.handle, ctypes.byref(params), int(mode), M, n_seq, _ptr(seg_off), _ptr(row_pos),
+                                         _ptr(active), _ptr(tok), _ptr(conf), _ptr(in_plan), _ptr(u), _ptr(commit),
+                                         _ptr(explore_row), _ptr(y), L, _stream())
+        _check(rc, "pvf_explore_commit")
+        return explore_row[:n_seq]
 
     # ------------------------------------------------------------------ planning-vocabulary calibration
     def new_calib_stats(self) -> Dict[str, torch.Tensor]:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libpvf.so")
-SOURCES = ["pvf_api.cu", "pvf_step.cu", "pvf_score.cu", "pvf_host.cu", "pvf_blocks.cu", "pvf_calib.cu"]
+SOURCES = ["pvf_api.cu", "pvf_step.cu", "pvf_score.cu", "pvf_host.cu", "pvf_blocks.cu", "pvf_calib.cu", "pvf_explore.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
 
