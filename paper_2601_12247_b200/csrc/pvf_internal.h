@@ -40,7 +40,7 @@ struct pvf_ctx {
 
 // Work split of pvf_score for M rows on n_sm SMs (see pvf_score.cu).
 struct pvf_score_geometry {
-    int m_tiles;     // ceil(M / 128)
+    int m_tiles;     // ceil(M / 128) row tiles
     int units;       // ceil(V / 16): vocabulary granules
     int mb;          // row tiles processed concurrently (one wave)
     int splits;      // vocabulary ranges per row tile = partial states per row
@@ -48,6 +48,8 @@ struct pvf_score_geometry {
     int ctas;        // mb * splits
     int a_rows;      // rows of the hidden-state TMA box
     int streaming;   // 1: at most 32 rows, handled by the swapped-operand streaming kernel
+    int paired;      // 1: more than 128 rows, handled by the paired (cta_group::2) kernel; then m_tiles counts
+                     //    256-row tiles, units granules of 32 entries, mb / splits pairs of blocks
 };
 pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm);
 size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm);
@@ -79,6 +81,32 @@ static inline cudaError_t pvf_launch(void (*kernel)(KArgs...), dim3 grid, dim3 b
     cfg.numAttrs = 0;
 #else
     cfg.numAttrs = 1;
+#endif
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// The same for a kernel whose blocks form clusters of two along x (grid.x even).
+template <typename... KArgs, typename... Args>
+static inline cudaError_t pvf_launch_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                              cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+#ifdef PVF_NO_PDL
+    cfg.numAttrs = 1;
+#else
+    cfg.numAttrs = 2;
 #endif
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }

@@ -195,15 +195,21 @@ def test_config2_sampled_rows_and_decisions_on_gpu_scores(llada):
 
 
 def test_second_model_shape_sampled():
-    # Dream-7B-like LM head: 56 k-panels, 9504 vocabulary granules (64.2 per block): both kernels
+    # Dream-7B-like LM head: 56 k-panels, 9504 vocabulary granules (64.2 per block): all three kernels
     V, D = synth.DREAM_VOCAB, synth.DREAM_HIDDEN
     w_bits = synth.make_w(1005, V, D)
     plan = synth.make_plan_ids(1005, V, 2048)
     ctx = make_ctx(w_bits, plan, 512, 8, 8)
-    for variant, sample in (("a", np.array([0, 1, 15, 16, 30, 31])), ("b", np.array([0, 127, 128, 129, 255]))):
-        st = synth.config1(variant, stress=True, w_bits=w_bits, vocab=V, hidden=D)
-        assert ctx.score_kernel_name(st.n_rows) == ("pvf_score_stream_kernel" if variant == "a" else "pvf_score_gemm_kernel")
-        sampled_parity(ctx, st, w_bits, plan, sample)
+    st = synth.config1("b", stress=True, w_bits=w_bits, vocab=V, hidden=D)
+    for rows, kernel, sample in ((32, "pvf_score_stream_kernel", np.array([0, 1, 15, 16, 30, 31])),
+                                 (100, "pvf_score_gemm_kernel", np.array([0, 31, 32, 64, 99])),
+                                 (256, "pvf_score_gemm_pair_kernel", np.array([0, 127, 128, 129, 255]))):
+        assert ctx.score_kernel_name(rows) == kernel
+        got = to_np(ctx.score(upload_bits(st.h_bits[:rows])))
+        torch.cuda.synchronize()
+        assert ctx.last_status() == 0
+        check_score_properties(got, V, plan)
+        check_score(got, oscore.score(w_bits, st.h_bits[sample], plan), V, plan, rows=sample)
     ctx.close()
 
 
