@@ -40,6 +40,7 @@ UNIT = "positions/s"
 # per-pass traffic by their number of passes over W ("waves").
 NCU_TRAFFIC_STREAM_LAUNCH = 1.04074e9
 NCU_TRAFFIC_GEMM_PER_WAVE = 1.244e9
+NCU_TRAFFIC_PAIR_PER_WAVE = 1.0497e9
 
 
 def load_peaks():
@@ -306,6 +307,8 @@ def run_ours(args):
         traffic = NCU_TRAFFIC_STREAM_LAUNCH
     elif kernels == ["pvf_score_gemm_kernel"] and NCU_TRAFFIC_GEMM_PER_WAVE is not None:
         traffic = NCU_TRAFFIC_GEMM_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
+    elif kernels == ["pvf_score_gemm_pair_kernel"] and NCU_TRAFFIC_PAIR_PER_WAVE is not None:
+        traffic = NCU_TRAFFIC_PAIR_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
     else:
         traffic = None
     roof.update(traffic=traffic, kernel="+".join(kernels), launches=n_gemm, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
