@@ -116,6 +116,12 @@ int pvf_last_status(pvf_ctx *ctx, int32_t *status);
  */
 int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int32_t *waves, int32_t *launches);
 
+/* The same plan from shapes alone (no context, no device): n_sm = number of SMs to plan for.  `kernel` (may be
+ * NULL) receives 0 for the streaming kernel, 1 for the 128-row GEMM kernel, 2 for the paired kernel; `row_tiles`
+ * the number of row tiles (256 rows in the paired kernel, else 128) and `tiles_per_wave` how many are in flight. */
+int pvf_score_plan_for_shape(int32_t vocab, int32_t hidden, int32_t n_sm, int32_t M, int32_t *ctas, int32_t *splits,
+                             int32_t *waves, int32_t *kernel, int32_t *row_tiles, int32_t *tiles_per_wave);
+
 /* Name of the projection kernel pvf_score launches for M rows (for profiler filters and reports):
  * "pvf_score_stream_kernel" up to 32 rows (vocabulary on the accumulator lanes, rows on its columns),
  * "pvf_score_gemm_kernel" above (rows on the lanes).  NULL on an invalid argument. */
@@ -306,6 +312,11 @@ int pvf_working_set(pvf_ctx *ctx, const int32_t *y, int32_t n_seq, int32_t L, in
  *                            max_rows * (2 * hidden + 40) bytes)
  *   pvf_attach_host_staging  hand the context a 256-byte-aligned device buffer of that size (kept until
  *                            replaced; NULL detaches).  Without it the two calls return PVF_ERR_WORKSPACE.
+ *   pvf_host_bounce_bytes    bytes of PINNED HOST memory for the optional bounce buffer of this shape
+ *   pvf_attach_host_bounce   hand the context such a buffer (kept until replaced; NULL detaches).  With it, the
+ *                            small input arrays travel as one host-to-device copy and all outputs of a call as
+ *                            one device-to-host copy into the buffer, from which they are copied to the output
+ *                            pointers (which then need not be pinned); without it every array is copied on its own.
  *   pvf_draft_step_host      pvf_score + pvf_commit + pvf_select_drafts on hidden_host[M][hidden]; outputs
  *                            as in those calls.  The device copies stay in the staging buffer.
  *   pvf_verify_step_host     pvf_score on hidden_v_host[Mv][hidden] + pvf_verify, continuing the draft
@@ -314,6 +325,8 @@ int pvf_working_set(pvf_ctx *ctx, const int32_t *y, int32_t n_seq, int32_t L, in
  */
 size_t pvf_host_staging_bytes(const pvf_shape *shape);
 int pvf_attach_host_staging(pvf_ctx *ctx, void *staging, size_t bytes);
+size_t pvf_host_bounce_bytes(const pvf_shape *shape);
+int pvf_attach_host_bounce(pvf_ctx *ctx, void *pinned_host, size_t bytes);
 int pvf_draft_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hidden_host, int32_t M, int32_t n_seq,
                         const int32_t *seg_off_host, const int32_t *row_pos_host, const uint8_t *active_host,
                         int32_t *tok_host, float *conf_host, float *ent_host, uint8_t *in_plan_host,

@@ -70,6 +70,8 @@ def load() -> ctypes.CDLL:
         lib.pvf_last_status.argtypes = [vp, ctypes.POINTER(i32)]; lib.pvf_last_status.restype = ctypes.c_int
         lib.pvf_set_score_events.argtypes = [vp, vp, vp]; lib.pvf_set_score_events.restype = ctypes.c_int
         lib.pvf_score_plan.argtypes = [vp, i32] + [ctypes.POINTER(i32)] * 4; lib.pvf_score_plan.restype = ctypes.c_int
+        lib.pvf_score_plan_for_shape.argtypes = [i32] * 4 + [ctypes.POINTER(i32)] * 6
+        lib.pvf_score_plan_for_shape.restype = ctypes.c_int
         lib.pvf_score_kernel_name.argtypes = [vp, i32]; lib.pvf_score_kernel_name.restype = ctypes.c_char_p
         lib.pvf_score.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]; lib.pvf_score.restype = ctypes.c_int
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
@@ -86,6 +88,8 @@ def load() -> ctypes.CDLL:
         lib.pvf_working_set.restype = ctypes.c_int
         lib.pvf_host_staging_bytes.argtypes = [ps]; lib.pvf_host_staging_bytes.restype = sz
         lib.pvf_attach_host_staging.argtypes = [vp, vp, sz]; lib.pvf_attach_host_staging.restype = ctypes.c_int
+        lib.pvf_host_bounce_bytes.argtypes = [ps]; lib.pvf_host_bounce_bytes.restype = sz
+        lib.pvf_attach_host_bounce.argtypes = [vp, vp, sz]; lib.pvf_attach_host_bounce.restype = ctypes.c_int
         lib.pvf_draft_step_host.argtypes = [vp, pp, vp, i32, i32] + [vp] * 14 + [vp]; lib.pvf_draft_step_host.restype = ctypes.c_int
         lib.pvf_verify_step_host.argtypes = [vp, pp, vp, i32] + [vp] * 5 + [vp]; lib.pvf_verify_step_host.restype = ctypes.c_int
         lib.pvf_score_static.argtypes = [vp, i32, i32, vp, i32, vp, vp, vp, vp, vp, vp]; lib.pvf_score_static.restype = ctypes.c_int
@@ -102,6 +106,14 @@ def default_params() -> pvf_params:
     p = pvf_params()
     load().pvf_default_params(ctypes.byref(p))
     return p
+
+
+def score_plan_for_shape(vocab: int, hidden: int, n_sm: int, M: int) -> Dict[str, int]:
+    """pvf_score_plan_for_shape: the work split pvf_score would use, computed on the host (no GPU needed)."""
+    v = [ctypes.c_int32() for _ in range(6)]
+    _check(load().pvf_score_plan_for_shape(int(vocab), int(hidden), int(n_sm), int(M), *[ctypes.byref(x) for x in v]),
+           "pvf_score_plan_for_shape")
+    return dict(zip(("ctas", "splits", "waves", "kernel", "row_tiles", "tiles_per_wave"), (x.value for x in v)))
 
 
 def default_calib_params() -> pvf_calib_params:
@@ -188,13 +200,21 @@ class Context:
         return name.decode()
 
     # ------------------------------------------------------------------ host-buffer variants
-    def attach_host_staging(self):
-        """Allocate the device staging buffer of the host-buffer calls and hand it to the context."""
+    def attach_host_staging(self, bounce: bool = True):
+        """Allocate the device staging buffer of the host-buffer calls (and, with ``bounce``, the pinned host
+        bounce buffer that packs their copies) and hand them to the context."""
         nbytes = self.lib.pvf_host_staging_bytes(ctypes.byref(self.shape))
         self.staging = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
         off = (-self.staging.data_ptr()) % 256
         _check(self.lib.pvf_attach_host_staging(self.handle, ctypes.c_void_p(self.staging.data_ptr() + off), nbytes),
                "pvf_attach_host_staging")
+        if bounce:
+            hbytes = self.lib.pvf_host_bounce_bytes(ctypes.byref(self.shape))
+            self.bounce = torch.empty(hbytes, dtype=torch.uint8).pin_memory()
+            _check(self.lib.pvf_attach_host_bounce(self.handle, ctypes.c_void_p(self.bounce.data_ptr()), hbytes),
+                   "pvf_attach_host_bounce")
+        else:
+            _check(self.lib.pvf_attach_host_bounce(self.handle, None, 0), "pvf_attach_host_bounce")
 
     def draft_step_host(self, params: pvf_params, hidden_host: torch.Tensor, seg_off: torch.Tensor, row_pos: torch.Tensor,
                         active: Optional[torch.Tensor], out: Dict[str, torch.Tensor]):

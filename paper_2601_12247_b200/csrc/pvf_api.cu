@@ -108,6 +108,7 @@ int pvf_create(pvf_ctx **out, const pvf_shape *shape, const void *w_head,
     ctx->ev_stop = nullptr;
     ctx->staging = nullptr;
     ctx->staging_bytes = 0;
+    ctx->bounce = nullptr;
     ctx->host_rows = ctx->host_seqs = ctx->host_budget = 0;
     ctx->host_active = false;
 

@@ -34,6 +34,7 @@ struct pvf_ctx {
     cudaEvent_t ev_start, ev_stop;   // optional timing hook around the GEMM kernel
     uint8_t *staging;                // optional device staging of the host-buffer entry points
     size_t staging_bytes;
+    uint8_t *bounce;                 // optional pinned host mirror of the staging's small arrays (one copy per direction)
     int32_t host_rows, host_seqs, host_budget;   // shape of the draft half the staging currently holds
     bool host_active;
 };

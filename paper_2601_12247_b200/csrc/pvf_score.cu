@@ -1323,6 +1323,20 @@ int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int3
     return PVF_OK;
 }
 
+int pvf_score_plan_for_shape(int32_t vocab, int32_t hidden, int32_t n_sm, int32_t M, int32_t *ctas, int32_t *splits,
+                             int32_t *waves, int32_t *kernel, int32_t *row_tiles, int32_t *tiles_per_wave)
+{
+    if (vocab <= 0 || hidden <= 0 || n_sm <= 0 || M <= 0) return PVF_ERR_INVALID;
+    const pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden, n_sm);
+    if (ctas) *ctas = g.ctas;
+    if (splits) *splits = g.splits;
+    if (waves) *waves = g.waves;
+    if (kernel) *kernel = g.streaming ? 0 : (g.paired ? 2 : 1);
+    if (row_tiles) *row_tiles = g.m_tiles;
+    if (tiles_per_wave) *tiles_per_wave = g.mb;
+    return PVF_OK;
+}
+
 const char *pvf_score_kernel_name(pvf_ctx *ctx, int32_t M)
 {
     if (!ctx || M <= 0 || M > ctx->shape.max_rows) return nullptr;

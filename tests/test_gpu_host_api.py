@@ -9,8 +9,8 @@ from gpu_util import make_ctx, params_of, t_i32, t_u8, to_np, upload_bits
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("stress,pinned", [(False, True), (True, False)])
-def test_host_step_equals_device_step(stress, pinned):
+@pytest.mark.parametrize("stress,pinned,bounce", [(False, True, True), (True, False, True), (True, True, False)])
+def test_host_step_equals_device_step(stress, pinned, bounce):
     w = synth.make_w(2002, 8192, 256)
     st = synth.config2(stress=stress, w_bits=w, vocab=8192, hidden=256)
     ctx = make_ctx(w, st.plan_ids, 16384, 64, 16)
@@ -32,7 +32,7 @@ def test_host_step_equals_device_step(stress, pinned):
         ctx.draft_step_host(prm, binding.bf16_from_bits(st.h_bits, "cpu"), torch.from_numpy(st.seg_off),
                             torch.from_numpy(st.row_pos), None, {})
     assert e.value.code == binding.PVF_ERR_WORKSPACE
-    ctx.attach_host_staging()
+    ctx.attach_host_staging(bounce=bounce)
     hb = binding.host_buffers(st.n_rows, st.n_seq, K, Mv, pinned=pinned)
     mk = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
     ctx.draft_step_host(prm, mk(binding.bf16_from_bits(st.h_bits, "cpu")), mk(torch.from_numpy(st.seg_off)),
