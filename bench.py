@@ -39,7 +39,7 @@ UNIT = "positions/s"
 # streaming kernel's config-1a launch is captured as is; launches of the GEMM kernel scale the captured
 # per-pass traffic by their number of passes over W ("waves").
 NCU_TRAFFIC_STREAM_LAUNCH = 1.04074e9
-NCU_TRAFFIC_GEMM_PER_WAVE = 1.244e9
+NCU_TRAFFIC_GEMM_PER_WAVE = 1.162e9
 NCU_TRAFFIC_PAIR_PER_WAVE = 1.0497e9
 
 
