@@ -12,32 +12,8 @@
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-
-__device__ __forceinline__ int block_sum(int v, int *scratch)
-{
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    int t = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += scratch[w];
-    return t;
-}
-
-__device__ __forceinline__ int block_min(int v, int *scratch)
-{
-    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    int t = scratch[0];
-#pragma unroll
-    for (int w = 1; w < kWarps; ++w) t = min(t, scratch[w]);
-    return t;
-}
+constexpr int kThreads = kPvfBlockThreads;
+constexpr int kWarps = kPvfBlockWarps;
 
 // Position range [lo, hi) that holds B_t of one sequence (empty when the sequence is finished), and
 // whether the next block was revealed.  Every thread of the block returns the same values.
@@ -47,13 +23,13 @@ __device__ __forceinline__ void working_range(const int32_t *__restrict__ yb, in
     int first = L;
     for (int i = threadIdx.x; i < L; i += kThreads)
         if (yb[i] == mask_id) { first = i; break; }            // a thread's positions ascend
-    first = block_min(first, scratch);
+    first = pvf_block_min(first, scratch);
     if (first >= L) { *lo = 0; *hi = 0; *expanded = 0; return; }
     const int k = first / S;                                   // k_t, 0-based
     const int b0 = k * S, b1 = min(b0 + S, L);
     int n_active = 0;                                          // |M_t^active|
     for (int i = b0 + threadIdx.x; i < b1; i += kThreads) n_active += yb[i] == mask_id ? 1 : 0;
-    n_active = block_sum(n_active, scratch);
+    n_active = pvf_block_sum(n_active, scratch);
     const int reveal = (n_active <= n_sparse && b1 < L) ? 1 : 0;
     *lo = b0;
     *hi = reveal ? min(b1 + S, L) : b1;                        // B_t = M_active, or M_active + I_{k_t+1}
@@ -74,7 +50,7 @@ pvf_working_count_kernel(const int32_t *__restrict__ y, int n_seq, int L, int S,
     working_range(yb, L, S, n_sparse, mask_id, s_int, &lo, &hi, &ex);
     int n = 0;
     for (int i = lo + threadIdx.x; i < hi; i += kThreads) n += yb[i] == mask_id ? 1 : 0;
-    n = block_sum(n, s_int);
+    n = pvf_block_sum(n, s_int);
     if (threadIdx.x == 0) {
         seg_off[b + 1] = n;                                    // a count for now
         if (expanded) expanded[b] = (uint8_t)ex;
@@ -120,24 +96,14 @@ pvf_working_fill_kernel(const int32_t *__restrict__ y, int L, int S, int n_spars
     const int32_t *yb = y + (size_t)b * L;
     int lo, hi, ex;
     working_range(yb, L, S, n_sparse, mask_id, s_int, &lo, &hi, &ex);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int out = seg_off[b];
     for (int c0 = lo; c0 < hi; c0 += kThreads) {               // block-uniform trip count
         const int i = c0 + threadIdx.x;
         const bool masked = i < hi && yb[i] == mask_id;
-        const unsigned ballot = __ballot_sync(0xffffffffu, masked);
-        __syncthreads();
-        if (lane == 0) s_int[warp] = __popc(ballot);
-        __syncthreads();
-        int before = 0, all = 0;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const int c = s_int[w];
-            if (w < warp) before += c;
-            all += c;
-        }
+        int all;
+        const int rank = pvf_block_rank(masked, s_int, &all);
         if (masked) {
-            const int m = out + before + __popc(ballot & ((1u << lane) - 1u));
+            const int m = out + rank;
             row_pos[m] = i;
             if (row_seq) row_seq[m] = b;
             if (active) active[m] = 1;

@@ -8,20 +8,8 @@
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-
-__device__ __forceinline__ int block_sum(int v, int *scratch)
-{
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    int t = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += scratch[w];
-    return t;
-}
+constexpr int kThreads = kPvfBlockThreads;
+constexpr int kWarps = kPvfBlockWarps;
 
 __global__ void __launch_bounds__(kThreads)
 pvf_explore_kernel(const int32_t *__restrict__ seg_off, const int32_t *__restrict__ row_pos,
@@ -44,8 +32,8 @@ pvf_explore_kernel(const int32_t *__restrict__ seg_off, const int32_t *__restric
         n_all += el ? 1 : 0;
         n_plan += (el && planning && in_plan[m]) ? 1 : 0;
     }
-    n_all = block_sum(n_all, s_int);
-    n_plan = block_sum(n_plan, s_int);
+    n_all = pvf_block_sum(n_all, s_int);
+    n_plan = pvf_block_sum(n_plan, s_int);
     const bool use_plan = planning && n_plan > 0;
     const int n = use_plan ? n_plan : n_all;
     if (n == 0) {

@@ -113,6 +113,55 @@ static inline cudaError_t pvf_launch_cluster2(void (*kernel)(KArgs...), dim3 gri
 }
 #endif
 
+// Block-wide helpers of the one-block-per-sequence kernels (256 threads; `scratch` holds one entry per warp).
+#ifdef __CUDACC__
+constexpr int kPvfBlockThreads = 256;
+constexpr int kPvfBlockWarps = kPvfBlockThreads / 32;
+
+__device__ __forceinline__ int pvf_block_sum(int v, int *scratch)
+{
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();                               // scratch may still be read from a previous call
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int t = 0;
+#pragma unroll
+    for (int w = 0; w < kPvfBlockWarps; ++w) t += scratch[w];
+    return t;
+}
+
+__device__ __forceinline__ int pvf_block_min(int v, int *scratch)
+{
+    for (int o = 16; o > 0; o >>= 1) v = min(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int t = scratch[0];
+#pragma unroll
+    for (int w = 1; w < kPvfBlockWarps; ++w) t = min(t, scratch[w]);
+    return t;
+}
+
+// Exclusive prefix of a 0/1 flag over the block, in thread order; *total gets the block's count.
+__device__ __forceinline__ int pvf_block_rank(bool flag, int *scratch, int *total)
+{
+    const unsigned ballot = __ballot_sync(0xffffffffu, flag);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) scratch[warp] = __popc(ballot);
+    __syncthreads();
+    int before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < kPvfBlockWarps; ++w) {
+        const int c = scratch[w];
+        if (w < warp) before += c;
+        all += c;
+    }
+    *total = all;
+    return before + __popc(ballot & ((1u << lane) - 1u));
+}
+#endif
+
 static inline size_t pvf_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 #endif

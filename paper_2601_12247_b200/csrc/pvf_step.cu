@@ -5,20 +5,8 @@
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kWarps = kThreads / 32;
-
-__device__ __forceinline__ int block_sum(int v, int *scratch)
-{
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    __syncthreads();                               // scratch may still be read from a previous call
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    int t = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += scratch[w];
-    return t;
-}
+constexpr int kThreads = kPvfBlockThreads;
+constexpr int kWarps = kPvfBlockWarps;
 
 __device__ __forceinline__ unsigned long long block_max(unsigned long long v, unsigned long long *scratch)
 {
@@ -33,25 +21,6 @@ __device__ __forceinline__ unsigned long long block_max(unsigned long long v, un
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) t = scratch[w] > t ? scratch[w] : t;
     return t;
-}
-
-// Exclusive prefix of a 0/1 flag over the block, in thread order; *total gets the block's count.
-__device__ __forceinline__ int block_rank(bool flag, int *scratch, int *total)
-{
-    const unsigned ballot = __ballot_sync(0xffffffffu, flag);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    __syncthreads();
-    if (lane == 0) scratch[warp] = __popc(ballot);
-    __syncthreads();
-    int before = 0, all = 0;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) {
-        const int c = scratch[w];
-        if (w < warp) before += c;
-        all += c;
-    }
-    *total = all;
-    return before + __popc(ballot & ((1u << lane) - 1u));
 }
 
 // Sort key of a candidate: larger confidence first, then the lower position (rows of a sequence
@@ -92,7 +61,7 @@ pvf_commit_kernel(const int32_t *__restrict__ seg_off, const int32_t *__restrict
             best = k > best ? k : best;
         }
     }
-    int total = block_sum(count, s_int);
+    int total = pvf_block_sum(count, s_int);
     if (force_progress && total == 0) {
         best = block_max(best, s_key);
         if (best != 0) {
@@ -128,7 +97,7 @@ pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t 
     int before = 0;
     for (int m = threadIdx.x; m < r0; m += kThreads)
         before += ((active ? active[m] != 0 : true) && !commit[m]) ? 1 : 0;
-    const int rem_base = block_sum(before, s_int);
+    const int rem_base = pvf_block_sum(before, s_int);
 
     // R_b in position order, and the number of planning candidates.
     int n_rem = 0, n_plan = 0;
@@ -141,12 +110,12 @@ pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t 
             plan = rem && (any_token || in_plan[m]) && p >= tau_lo && p < tau_hi;  // P_t^plan
         }
         int chunk_total;
-        const int rank = block_rank(rem, s_int, &chunk_total);
+        const int rank = pvf_block_rank(rem, s_int, &chunk_total);
         if (rem) rem_rows[rem_base + n_rem + rank] = m;
         n_rem += chunk_total;
         n_plan += plan ? 1 : 0;
     }
-    n_plan = block_sum(n_plan, s_int);
+    n_plan = pvf_block_sum(n_plan, s_int);
 
     int kt = 0, rt = 0;
     if (K > 0 && n_plan > 0) {
@@ -175,7 +144,7 @@ pvf_select_kernel(int n_seq, const int32_t *__restrict__ seg_off, const uint8_t 
             const int m = c0 + threadIdx.x;
             const bool ok = m < r1 && (active ? active[m] != 0 : true) && !commit[m] && conf[m] >= tau_ar;
             int chunk_total;
-            const int rank = block_rank(ok, s_int, &chunk_total);
+            const int rank = pvf_block_rank(ok, s_int, &chunk_total);
             if (ok && kt + rank < K) draft_rows[(size_t)b * K + kt + rank] = m;
             kt += chunk_total;
         }

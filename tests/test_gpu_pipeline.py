@@ -194,6 +194,15 @@ def test_config2_sampled_rows_and_decisions_on_gpu_scores(llada):
         check_score(gscv, oscore.score(w_bits, v.hv_bits[rows], plan), st.vocab, plan, rows=rows)
 
 
+def test_paired_kernel_two_waves_sampled(llada):
+    # 4096 rows: 16 tiles of 256 rows, 8 in flight, 9 vocabulary ranges, 2 waves of the paired kernel
+    w_bits, plan, ctx = llada
+    st = synth.config3(w_bits=w_bits, n_seq=8)
+    assert st.n_rows == 4096 and ctx.score_kernel_name(4096) == "pvf_score_gemm_pair_kernel"
+    assert ctx.score_plan(4096)["waves"] == 2
+    sampled_parity(ctx, st, w_bits, plan, np.array([0, 127, 128, 255, 256, 2047, 2048, 2303, 2304, 4095]))
+
+
 def test_second_model_shape_sampled():
     # Dream-7B-like LM head: 56 k-panels, 9504 vocabulary granules (64.2 per block): all three kernels
     V, D = synth.DREAM_VOCAB, synth.DREAM_HIDDEN
