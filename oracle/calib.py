@@ -91,3 +91,61 @@ def filter_tokens(stats: Dict[str, np.ndarray], n_min: int, m_min: int, rho_ver:
         if r_ver >= rho and vig_hat >= gam:
             keep.append(v)
     return np.asarray(keep, dtype=np.int32)
+
+
+def calibrate(synth, w_bits, targets, seed: int, gen_len: int, block: int, tau_high: float, tau_cal_lo: float,
+              tau_cal_hi: float, budget: int, mask_id: int, max_steps: int = 100000, trace: bool = False) -> Dict:
+    """Calibration trajectory on synthetic hidden states (Appendix, "Calibration trajectory").
+
+    The canvas is decoded with the confidence-threshold base rule alone (forced progress as in the decode
+    loop).  At every step the candidates C_t^cal are measured -- one planning branch each, scored by the
+    generator's verification-pass hidden states -- and their events are added to the token statistics; the
+    branches are never committed.  Returns the statistics, the number of events and steps."""
+    from . import loop as oloop
+    from . import score as oscore
+    from . import step as ostep
+    n_seq = targets.shape[0]
+    vocab = w_bits.shape[0]
+    y = np.full((n_seq, gen_len), mask_id, dtype=np.int32)
+    stats = new_stats(vocab)
+    n_events = n_steps = 0
+    history = []
+    while (y == mask_id).any():
+        if n_steps >= max_steps:
+            raise RuntimeError("calibration loop did not terminate")
+        seq_ids, positions, seg_off = oloop.working_rows(y, mask_id, block)
+        frac = (y != mask_id).sum(axis=1) / float(gen_len)
+        h = synth.loop_hidden(w_bits, targets, seed, n_steps, 0, seq_ids, positions, frac)
+        sc = oscore.score(w_bits, h, None)
+        active = np.ones(len(positions), np.uint8)
+        cm = ostep.commit(sc["conf"], sc["tok"], seg_off, positions, active, tau_high, force_progress=True)
+        sel = ostep.select_drafts(sc["conf"], sc["tok"], sc["in_plan"], cm["commit"], seg_off, positions, active,
+                                  tau_cal_lo, tau_cal_hi, 0.0, budget, any_token=True, ar_fallback=False)
+        vb, vi, vc = [], [], []
+        for b in range(n_seq):
+            rem = sel["rem_rows"][sel["rem_off"][b]:sel["rem_off"][b + 1]]
+            if sel["n_drafts"][b] > 0:
+                for c in range(1 + int(sel["n_drafts"][b])):
+                    for m in rem:
+                        vb.append(b); vi.append(int(positions[m])); vc.append(c)
+        evs = []
+        scv = None
+        if vb:
+            hv = synth.loop_verify_hidden(w_bits, targets, seed, n_steps, np.asarray(vb, np.int32),
+                                          np.asarray(vi, np.int32), np.asarray(vc, np.int32), frac)
+            scv = oscore.score(w_bits, hv, None)
+            evs = events(sc["tok"], sel["rem_rows"], sel["rem_off"], sel["v_off"], sel["draft_rows"], sel["n_drafts"],
+                         sel["route"], scv["tok"], scv["conf"], scv["ent"], tau_high)
+            accumulate(stats, evs)
+            n_events += len(evs)
+        for m in range(len(positions)):                      # only the base set is committed
+            if cm["commit"][m]:
+                y[seq_ids[m], positions[m]] = sc["tok"][m]
+        if trace:
+            history.append(dict(positions=positions.copy(), seq_ids=seq_ids.copy(), score=sc, commit=cm, select=sel,
+                                score_v=scv, events=evs, y=y.copy()))
+        n_steps += 1
+    out = dict(stats=stats, n_events=n_events, steps=n_steps, y=y)
+    if trace:
+        out["history"] = history
+    return out

@@ -56,10 +56,16 @@ def working_rows(y: np.ndarray, mask_id: int, block: int, n_sparse: int = 0):
 
 
 def decode(synth, w_bits, plan_ids, targets, seed: int, gen_len: int, block: int, params: Dict,
-           mask_id: int, max_steps: int = 100000, trace: bool = False, n_sparse: int = 0) -> Dict:
-    """Run Algorithm 1 until no masks remain.  ``synth`` is the input-generator module."""
+           mask_id: int, max_steps: int = 100000, trace: bool = False, n_sparse: int = 0,
+           explore: str = "") -> Dict:
+    """Run Algorithm 1 until no masks remain.  ``synth`` is the input-generator module.
+
+    ``explore`` = "random" or "planning" runs the appendix's exploration loop instead ("Planning tokens
+    beyond high-confidence decoding"): every step commits the base set and then exactly one more token
+    from the closed confidence bin [tau_plan_lo, tau_plan_hi]; nothing is drafted or verified (the budget
+    is ignored).  The uniform draws come from the input generator."""
     n_seq = targets.shape[0]
-    K = int(params["budget"])
+    K = 0 if explore else int(params["budget"])
     y = np.full((n_seq, gen_len), mask_id, dtype=np.int32)
     steps_per_seq = np.zeros(n_seq, dtype=np.int32)
     scored_rows = 0
@@ -77,7 +83,12 @@ def decode(synth, w_bits, plan_ids, targets, seed: int, gen_len: int, block: int
                           force_progress=True)
         scored_rows += len(positions)
         final = cm["commit"]
-        sel = ver = None
+        sel = ver = exp = None
+        if explore:
+            exp = ostep.explore_commit(sc["conf"], sc["tok"], sc["in_plan"], cm["commit"], seg_off, positions, active,
+                                       params["tau_plan_lo"], params["tau_plan_hi"],
+                                       synth.loop_uniforms(seed, n_steps, n_seq), explore == "planning")
+            final = exp["commit"]
         if K > 0:
             sel = ostep.select_drafts(sc["conf"], sc["tok"], sc["in_plan"], cm["commit"], seg_off,
                                       positions, active, params["tau_plan_lo"], params["tau_plan_hi"],
@@ -105,7 +116,7 @@ def decode(synth, w_bits, plan_ids, targets, seed: int, gen_len: int, block: int
                 steps_per_seq[b] += 1
         if trace:
             history.append(dict(positions=positions.copy(), seq_ids=seq_ids.copy(), score=sc,
-                                commit=cm, select=sel, verify=ver, y=y.copy()))
+                                commit=cm, select=sel, verify=ver, explore=exp, y=y.copy()))
         n_steps += 1
     out = dict(y=y, steps=n_steps, steps_per_seq=steps_per_seq, scored_rows=scored_rows,
                tokens_per_forward=float(np.mean(gen_len / np.maximum(steps_per_seq, 1))))

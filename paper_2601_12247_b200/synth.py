@@ -41,6 +41,7 @@ TAG_SEQ = 11
 TAG_LOOP_AMP = 12
 TAG_LOOP_NOISE = 13
 TAG_PLAN_PICK = 14
+TAG_EXPLORE = 15
 
 LLADA_VOCAB = 126464
 LLADA_HIDDEN = 4096
@@ -375,3 +376,9 @@ def loop_verify_hidden(w_bits: np.ndarray, targets: np.ndarray, seed: int, step_
         tg[r] = t
         keys[r] = (step_no * 64 + 1 + c, b, i)
     return make_hidden_rows(w_bits, tg, am, seed, TAG_LOOP_NOISE, keys)
+
+
+def loop_uniforms(seed: int, step_no: int, n_seq: int) -> np.ndarray:
+    """One uniform number in [0, 1) per sequence for a loop step (float32): the random draws that the
+    exploration variants take as an input."""
+    return np.array([_rng(seed, TAG_EXPLORE, step_no, b).random() for b in range(n_seq)], dtype=np.float32)

@@ -151,3 +151,29 @@ def test_calibration_candidates_are_the_band_without_vocabulary_filter():
     sel3 = ostep.select_drafts(conf, tok, in_plan, cm["commit"], seg, pos, act, 0.5, 0.6, 0.1, 8,
                                any_token=True, ar_fallback=False)
     assert sel3["route"][0] == 0 and sel3["n_drafts"][0] == 0 and sel3["v_off"][-1] == 0
+
+
+def test_calibration_trajectory_is_threshold_decoding_plus_measurement():
+    from oracle import loop as oloop
+    from paper_2601_12247_b200 import synth
+    V, D, B, L, S, seed, mask = 1024, 64, 3, 64, 32, 1004, 1023
+    w = synth.make_w(seed, V, D)
+    plan = synth.make_plan_ids(seed, V, 128)
+    tg = synth.loop_targets(seed, V, B, L, plan, 0.5, avoid=mask)
+    r = ocal.calibrate(synth, w, tg, seed, L, S, 0.9, 0.15, 0.6, 8, mask, trace=True)
+    # the trajectory itself is confidence-threshold decoding: measuring commits nothing
+    base = oloop.decode(synth, w, plan, tg, seed, L, S, dict(tau_high=0.9, tau_plan_lo=0.2, tau_plan_hi=0.65,
+                                                             tau_ar_lo=0.1, budget=0), mask)
+    assert np.array_equal(r["y"], base["y"]) and r["steps"] == base["steps"]
+    st = r["stats"]
+    assert r["n_events"] > 0 and st["n"].sum() == r["n_events"]
+    assert np.all(st["sum_a"] <= st["m"]) and np.all(st["m"] <= st["n"])
+    seen = set()
+    for h in r["history"]:
+        assert (h["select"]["route"] != 2).all()
+        for e in h["events"]:
+            assert abs(e["dH"]) <= np.log(V) + 1e-9
+            seen.add(e["token"])
+    assert set(np.nonzero(st["n"])[0].tolist()) == seen
+    keep = ocal.filter_tokens(st, 1, 1, 0.5, -100.0)
+    assert set(keep.tolist()) <= seen

@@ -100,3 +100,25 @@ def test_early_cross_block_revelation_loop_terminates_and_never_skips_ahead():
                 new = np.nonzero((h["y"][b] != MASK) & (prev[b] == MASK))[0]
                 assert np.all(new < (k + 2) * S)
         prev = h["y"]
+
+
+def test_exploration_loops_commit_one_extra_token_per_step():
+    w, plan, tg = setup()
+    base = oloop.decode(synth, w, plan, tg, SEED, L, S, dict(P, budget=0), MASK)
+    for mode in ("random", "planning"):
+        r = oloop.decode(synth, w, plan, tg, SEED, L, S, P, MASK, trace=True, explore=mode)
+        assert not (r["y"] == MASK).any()
+        assert r["steps_per_seq"].sum() <= base["steps_per_seq"].sum()      # never slower than threshold decoding
+        extra_total = 0
+        for h in r["history"]:
+            ex = h["explore"]
+            extra = (ex["commit"].astype(int) - h["commit"]["commit"].astype(int))
+            assert extra.min() >= 0 and h["select"] is None and h["verify"] is None
+            for b in range(B):
+                rows = np.nonzero(h["seq_ids"] == b)[0]
+                assert extra[rows].sum() == (1 if ex["explore_row"][b] >= 0 else 0)
+                if ex["explore_row"][b] >= 0:
+                    p = h["score"]["conf"][ex["explore_row"][b]]
+                    assert float(np.float32(P["tau_plan_lo"])) <= p <= float(np.float32(P["tau_plan_hi"]))
+            extra_total += int(extra.sum())
+        assert extra_total > 0
