@@ -27,13 +27,15 @@ from . import binding, synth
 
 def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: int, gen_len: int, block: int,
            params: Dict, mask_id: int, max_steps: int = 100000,
-           on_step: Optional[Callable[[int, Dict], None]] = None, n_sparse: int = 0) -> Dict:
+           on_step: Optional[Callable[[int, Dict], None]] = None, n_sparse: int = 0, explore: str = "") -> Dict:
     """Run the loop until no masks remain.  ``params`` holds tau_high, tau_plan_lo, tau_plan_hi, tau_ar_lo
     and budget; ``n_sparse`` is the early cross-block threshold N_s (Eq. 4; 0 = strict block order).
+    ``explore`` = "random" / "planning" runs the appendix's exploration loop instead (base commit plus one
+    token from the closed bin [tau_plan_lo, tau_plan_hi] per step, no drafts, no verification).
     Returns y, step counts, scored rows and kernel times."""
     dev = ctx.device
     n_seq = targets.shape[0]
-    K = int(params["budget"])
+    K = 0 if explore else int(params["budget"])
     prm = binding.make_params(params["tau_high"], params["tau_plan_lo"], params["tau_plan_hi"], params["tau_ar_lo"],
                               K, binding.PVF_FORCE_PROGRESS)
     y_dev = torch.full((n_seq, gen_len), mask_id, dtype=torch.int32, device=dev)
@@ -56,8 +58,12 @@ def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: 
         e[0].record()
         sc = ctx.score(h)
         cm = ctx.commit(prm, seg, pos, None, sc["tok"], sc["conf"], y=y_dev)
-        sel = ver = scv = None
+        sel = ver = scv = exp_row = None
         hv_bits = None
+        if explore:
+            u = torch.from_numpy(synth.loop_uniforms(seed, n_steps, n_seq)).to(dev)
+            mode = binding.PVF_EXPLORE_PLANNING if explore == "planning" else binding.PVF_EXPLORE_RANDOM
+            exp_row = ctx.explore_commit(prm, mode, seg, pos, None, sc["tok"], sc["conf"], sc["in_plan"], u, cm["commit"], y=y_dev)
         if K > 0:
             sel = ctx.select_drafts(prm, seg, pos, None, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
         e[1].record()
@@ -86,7 +92,7 @@ def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: 
         steps_per_seq += (np.diff(seg_off) > 0).astype(np.int32)
         if on_step is not None:
             on_step(n_steps, dict(seq_ids=seq_ids, positions=positions, seg_off=seg_off, h_bits=h_bits, hv_bits=hv_bits,
-                                  score=sc, commit=cm, select=sel, score_v=scv, verify=ver, y=y.copy()))
+                                  score=sc, commit=cm, select=sel, score_v=scv, verify=ver, explore_row=exp_row, y=y.copy()))
         n_steps += 1
     status = ctx.last_status()
     return dict(y=y, steps=n_steps, steps_per_seq=steps_per_seq, scored_rows=scored_rows, status=status,
@@ -105,6 +111,7 @@ def main():
     ap.add_argument("--n-plan", type=int, default=2048)
     ap.add_argument("--q-plan", type=float, default=0.0, help="fraction of targets drawn from the planning ids")
     ap.add_argument("--n-sparse", type=int, default=0, help="early cross-block threshold N_s (Eq. 4)")
+    ap.add_argument("--explore", action="store_true", help="also run the Random / Planning exploration loops")
     ap.add_argument("--seed", type=int, default=1004)
     args = ap.parse_args()
     dev = torch.device("cuda:0")
@@ -121,6 +128,12 @@ def main():
         out[name] = dict(steps=r["steps"], mean_steps_per_sequence=float(r["steps_per_seq"].mean()),
                          tokens_per_forward=r["tokens_per_forward"], scored_rows=r["scored_rows"],
                          kernel_ms_per_step=r["kernel_ms_per_step"], status=r["status"])
+    if args.explore:
+        for mode in ("random", "planning"):
+            r = decode(ctx, w_bits, targets, args.seed, args.gen_len, args.block, p, args.vocab - 128, explore=mode)
+            out["explore_" + mode] = dict(steps=r["steps"], mean_steps_per_sequence=float(r["steps_per_seq"].mean()),
+                                          tokens_per_forward=r["tokens_per_forward"], scored_rows=r["scored_rows"],
+                                          kernel_ms_per_step=r["kernel_ms_per_step"], status=r["status"])
     out["config"] = dict(vocab=args.vocab, hidden=args.hidden, n_seq=args.n_seq, gen_len=args.gen_len, block=args.block,
                          budget=args.budget, q_plan=args.q_plan, n_sparse=args.n_sparse, data="synthetic")
     print(json.dumps(out))

@@ -89,3 +89,77 @@ def test_loop_llada_shape_two_sequences_sampled_rows():
     base = decode_loop.decode(ctx, w, tg, seed, L, S, dict(p, budget=0), V - 128)
     assert got["steps_per_seq"].sum() <= base["steps_per_seq"].sum() + 2
     ctx.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("mode", ["random", "planning"])
+def test_exploration_loop_state_by_state(mode):
+    V, D, B, L, S, seed = 4096, 256, 4, 64, 32, 1004
+    w = synth.make_w(seed, V, D)
+    plan = synth.make_plan_ids(seed, V, 256)
+    tg = synth.loop_targets(seed, V, B, L, plan, 0.5, avoid=V - 1)
+    p = dict(tau_high=0.9, budget=0, **synth.DEFAULT_BAND)
+    mask = V - 1
+    want = oloop.decode(synth, w, plan, tg, seed, L, S, p, mask, trace=True, explore=mode)
+    ctx = make_ctx(w, plan, B * S * 2, B, 1)
+    trace = []
+    got = decode_loop.decode(ctx, w, tg, seed, L, S, p, mask, on_step=lambda s, d: trace.append(
+        dict(d, commit_np=d["commit"]["commit"].cpu().numpy(), explore_np=d["explore_row"].cpu().numpy())), explore=mode)
+    assert got["status"] == 0 and not (got["y"] == mask).any()
+    n_same = 0
+    for g, o in zip(trace, want["history"]):
+        if fragile_step(o, p):
+            break
+        assert np.array_equal(g["positions"], o["positions"])
+        check_score(to_np(g["score"]), o["score"], V, plan)
+        assert np.array_equal(g["explore_np"], o["explore"]["explore_row"])
+        assert np.array_equal(g["commit_np"], o["explore"]["commit"])          # base commit plus the explored row
+        assert np.array_equal(g["y"], o["y"])
+        n_same += 1
+    assert n_same >= min(4, want["steps"])
+    if n_same == want["steps"]:
+        assert got["steps"] == want["steps"] and np.array_equal(got["y"], want["y"])
+    ctx.close()
+
+
+@pytest.mark.gpu
+def test_calibration_trajectory_matches_oracle():
+    from oracle import calib as ocal
+    from paper_2601_12247_b200 import calibrate
+    V, D, B, L, S, seed, K = 4096, 256, 4, 64, 32, 1006, 8
+    w = synth.make_w(seed, V, D)
+    pool = synth.make_plan_ids(seed, V, 24)
+    tg = synth.loop_targets(seed, V, B, L, pool, 1.0, avoid=V - 1)
+    mask = V - 1
+    cal = binding.default_calib_params()
+    cal.tau_cal_hi = 0.6                                     # a wider band than the paper's: more events in a tiny run
+    want = ocal.calibrate(synth, w, tg, seed, L, S, 0.9, cal.tau_cal_lo, cal.tau_cal_hi, K, mask, trace=True)
+    ctx = make_ctx(w, [], B * S * (2 + K), B, K)
+    trace = []
+    got = calibrate.calibrate(ctx, w, tg, seed, L, S, 0.9, cal, K, mask, on_step=lambda s, d: trace.append(d))
+    assert got["status"] == 0
+    taus = [0.9, cal.tau_cal_lo, cal.tau_cal_hi]
+    clean = True
+    for g, o in zip(trace, want["history"]):
+        bad = (o["score"]["gap"] < NEAR_TIE).any() or any((np.abs(o["score"]["conf"] - float(np.float32(t))) < FRAGILE).any() for t in taus)
+        if o["score_v"] is not None:
+            bad = bad or (o["score_v"]["gap"] < NEAR_TIE).any() or (np.abs(o["score_v"]["conf"] - float(np.float32(0.9))) < FRAGILE).any()
+        if bad:
+            clean = False
+            break
+        gs = to_np(g["select"])
+        for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+            assert np.array_equal(gs[k], o["select"][k]), k
+        if o["events"]:
+            vig = g["vig"].cpu().numpy()
+            for e in o["events"]:
+                assert abs(vig[e["seq"], e["j"] - 1] - e["VIG"]) <= 2e-3       # entropies within 1e-3 on both branches
+        assert np.array_equal(g["y"], o["y"])
+    assert want["n_events"] > 0
+    if clean:
+        st = to_np(got["stats"])
+        assert got["steps"] == want["steps"] and got["n_events"] == want["n_events"]
+        assert np.array_equal(st["n_v"], want["stats"]["n"]) and np.array_equal(st["m_v"], want["stats"]["m"])
+        assert np.array_equal(st["sum_a"], want["stats"]["sum_a"])
+        assert np.max(np.abs(st["sum_vig_q32"] / 2.0 ** 32 - want["stats"]["sum_vig"])) <= 2e-3 * max(1, want["n_events"])
+    ctx.close()
