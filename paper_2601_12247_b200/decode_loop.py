@@ -130,7 +130,8 @@ def main():
                          kernel_ms_per_step=r["kernel_ms_per_step"], status=r["status"])
     if args.explore:
         for mode in ("random", "planning"):
-            r = decode(ctx, w_bits, targets, args.seed, args.gen_len, args.block, p, args.vocab - 128, explore=mode)
+            r = decode(ctx, w_bits, targets, args.seed, args.gen_len, args.block, p, args.vocab - 128,
+                       n_sparse=args.n_sparse, explore=mode)
             out["explore_" + mode] = dict(steps=r["steps"], mean_steps_per_sequence=float(r["steps_per_seq"].mean()),
                                           tokens_per_forward=r["tokens_per_forward"], scored_rows=r["scored_rows"],
                                           kernel_ms_per_step=r["kernel_ms_per_step"], status=r["status"])
