@@ -259,6 +259,25 @@ __device__ __forceinline__ float fast_exp2(float x)
     return y;
 }
 
+// Barrier set-up shared by the three projection kernels (one thread): `issuers` threads commit every stage and
+// every accumulator, `drainers` epilogue threads release an accumulator.
+__device__ __forceinline__ void init_pipeline_barriers(SharedControl *ctl, int stages, int issuers, int drainers)
+{
+    for (int s = 0; s < stages; ++s) {
+        mbar_init(smem_u32(&ctl->full[s]), 1);
+        mbar_init(smem_u32(&ctl->empty[s]), issuers);
+    }
+    for (int b = 0; b < 2; ++b) {
+        mbar_init(smem_u32(&ctl->acc_full[b]), issuers);
+        mbar_init(smem_u32(&ctl->acc_empty[b]), drainers);
+    }
+    mbar_init(smem_u32(&ctl->drain), 1);
+    mbar_init(smem_u32(&ctl->drain2), 1);
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
 // ---------------------------------------------------------------------------------- work split
 // Vocabulary granules [u0, u1) of split q.
 __device__ __forceinline__ void split_range(int units, int splits, int q, int *u0, int *u1)
@@ -371,20 +390,7 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     const int n_tiles = split.n_tiles;                                   // vocabulary tiles per sweep
     const int k_steps = (args.num_kb + kPanels - 1) / kPanels;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
-            mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueThreads);
-        }
-        mbar_init(smem_u32(&ctl->drain), 1);
-        ctl->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
+    if (threadIdx.x == 0) init_pipeline_barriers(ctl, kStages, 1, kEpilogueThreads);
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.size[kWBoxSizes - 1]) : "memory");
@@ -652,20 +658,7 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     const int n_tiles = split.n_tiles;
     const int k_steps = args.num_kb;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kPairStages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), 1);
-            mbar_init(smem_u32(&ctl->acc_empty[b]), 2 * kEpilogueThreads);
-        }
-        mbar_init(smem_u32(&ctl->drain), 1);
-        ctl->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
+    if (threadIdx.x == 0) init_pipeline_barriers(ctl, kPairStages, 1, 2 * kEpilogueThreads);
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.size[kPairUnitsPerTile - 1]) : "memory");
@@ -888,21 +881,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     const int n_cols = args.M <= 16 ? 16 : 32;                           // MMA N: scored rows, padded
     const int k_steps = args.num_kb;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kStreamStages; ++s) {
-            mbar_init(smem_u32(&ctl->full[s]), 1);
-            mbar_init(smem_u32(&ctl->empty[s]), kStreamIssuers);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(smem_u32(&ctl->acc_full[b]), kStreamIssuers);
-            mbar_init(smem_u32(&ctl->acc_empty[b]), kEpilogueThreads);
-        }
-        mbar_init(smem_u32(&ctl->drain), 1);
-        mbar_init(smem_u32(&ctl->drain2), 1);
-        ctl->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
+    if (threadIdx.x == 0) init_pipeline_barriers(ctl, kStreamStages, kStreamIssuers, kEpilogueThreads);
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.size[kWBoxSizes - 1]) : "memory");
