@@ -15,7 +15,11 @@ with the CUDA library and never imports it.
 
 Pins (tests/test_oracle_*.py): closed forms (uniform row, identity weights), invariances,
 scipy's fp64 log_softmax on tiny shapes, brute-force argmax / top-k, a streaming recurrence
-versus the two-pass definition, hand-built verification cases and the step's invariants.
+versus the two-pass definition, hand-built verification cases and the step's invariants;
+hand-built canvases and an independent block rule for the working set; hand-computed
+information-gain events, a dictionary restatement of the token statistics and the filter's
+boundaries at the paper's printed thresholds; closed-bin edges and even-grid uniformity of
+the exploration variants.
 The paper prints no worked numeric example of a step, so parity with printed values is
 unpinned; its printed hyper-parameters (Table 5, Section 5.1) are pinned as defaults.
 """

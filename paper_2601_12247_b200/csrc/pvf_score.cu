@@ -1058,7 +1058,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
 // One warp per row: combines the row's `splits` partial states (ascending vocabulary ranges) in
 // fp64 and writes token, confidence, entropy and planning-vocabulary membership.
 __global__ void __launch_bounds__(256)
-pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int splits,
+pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int splits, int vocab,
                        const uint32_t *__restrict__ plan_bitmap, int32_t *__restrict__ tok,
                        float *__restrict__ conf, float *__restrict__ ent, uint8_t *__restrict__ in_plan)
 {
@@ -1097,6 +1097,9 @@ pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int splits,
         t += __shfl_xor_sync(0xffffffffu, t, o);
     }
     if (lane == 0) {
+        // A row of non-finite logits never sets a maximum: its outputs are unspecified, but the token stays a
+        // valid id and the bitmap lookup in bounds.
+        if ((unsigned)arg >= (unsigned)vocab) arg = 0;
         tok[row] = arg;
         conf[row] = (float)(1.0 / s);
         if (ent) ent[row] = (float)(log(s) - t / s);
@@ -1190,7 +1193,7 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
     if (timed && cudaEventRecord(ev_stop, s) != cudaSuccess) return PVF_ERR_CUDA;
     const int warps_per_block = 8;
     e = pvf_launch(pvf_score_merge_kernel, dim3((M + warps_per_block - 1) / warps_per_block), dim3(warps_per_block * 32), 0, s,
-                   (const float4 *)partials, M, g.splits, plan_bitmap, tok, conf, ent, in_plan);
+                   (const float4 *)partials, M, g.splits, V, plan_bitmap, tok, conf, ent, in_plan);
     return e == cudaSuccess ? PVF_OK : PVF_ERR_CUDA;
 }
 

@@ -113,3 +113,28 @@ def test_argument_errors_launch_nothing():
     torch.cuda.synchronize()
     assert ctx.last_status() == 0
     ctx.close()
+
+
+@pytest.mark.parametrize("M", [8, 100, 300])
+def test_non_finite_hidden_rows_stay_in_bounds_and_do_not_disturb_other_rows(M):
+    # rows holding NaN or Inf have unspecified outputs, but the call terminates, reports no error, returns valid
+    # token ids, and every other row is scored as if they were not there (all three kernels)
+    V, D = 5000, 200
+    pos = np.arange(M)
+    st = synth.build_step("nonfinite", 99, V, D, 64, [(pos, np.ones(M, np.uint8))], M, M,
+                          dict(tau_high=0.9, budget=4), amp_max=40.0 * (256.0 / D) ** 0.5)
+    h = st.h_bits.copy()
+    nan, inf, ninf = 0x7FC0, 0x7F80, 0xFF80                       # bf16 bit patterns
+    bad = [1, M // 2, M - 1]
+    h[bad[0], 3] = nan
+    h[bad[1], :] = inf
+    h[bad[2], 0] = ninf
+    ctx = make_ctx(st.w_bits, st.plan_ids, M)
+    got = to_np(ctx.score(upload_bits(h)))
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    assert np.all((got["tok"] >= 0) & (got["tok"] < V)) and np.all(got["in_plan"] <= 1)
+    good = np.setdiff1d(np.arange(M), bad)
+    want = oscore.score(st.w_bits, st.h_bits[good], st.plan_ids)
+    check_score(got, want, V, st.plan_ids, rows=good)
+    ctx.close()
