@@ -347,7 +347,7 @@ def run_ours(args):
                steps=n_e2e, ms_per_step=ms_e2e / n_e2e, api="pvf_draft_step_host + pvf_verify_step_host")
 
     # ---------------- CPU baseline: the oracle on the same step (rank 0, single-GPU runs only)
-    cpu = None
+    cpu = parity = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         from oracle import score as oscore
         from oracle import step as ostep
@@ -359,9 +359,21 @@ def run_ours(args):
             ocm = ostep.commit(osc["conf"], osc["tok"], st.seg_off, st.row_pos, st.active, p["tau_high"])
             ostep.select_drafts(osc["conf"], osc["tok"], osc["in_plan"], ocm["commit"], st.seg_off, st.row_pos,
                                 st.active, p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], K)
-        if rows_v:
-            oscore.score(st.w_bits, vp.hv_bits[:rows_v], st.plan_ids)
+        oscv = oscore.score(st.w_bits, vp.hv_bits[:rows_v], st.plan_ids) if rows_v else None
         dt = time.perf_counter() - t0
+        # parity of the step just timed against the same oracle results (outside the timed regions)
+        g = {k: v.cpu().numpy() for k, v in o_sc.items()}
+        near = osc["gap"] < 1e-3
+        parity = dict(rows=rows, max_conf_err=float(np.max(np.abs(g["conf"][:rows] - osc["conf"]))),
+                      max_ent_err=float(np.max(np.abs(g["ent"][:rows] - osc["ent"]))),
+                      near_tie_rows=int(near.sum()),
+                      token_mismatches_outside_near_ties=int((g["tok"][:rows][~near] != osc["tok"][~near]).sum()))
+        if oscv is not None:
+            gv = {k: v.cpu().numpy() for k, v in o_scv.items()}
+            nearv = oscv["gap"] < 1e-3
+            parity.update(verify_rows=rows_v, max_conf_err_verify=float(np.max(np.abs(gv["conf"][:rows_v] - oscv["conf"]))),
+                          near_tie_rows_verify=int(nearv.sum()),
+                          token_mismatches_outside_near_ties_verify=int((gv["tok"][:rows_v][~nearv] != oscv["tok"][~nearv]).sum()))
         frac = (rows + rows_v) / float(M + Mv)
         cpu = dict(value=M * frac / dt, unit=UNIT, cores=oscore.threads(), kind="oracle", seconds=dt,
                    sample="%d of %d draft-pass rows and %d of %d verification-pass rows of the same step, fp64 score%s"
@@ -380,7 +392,7 @@ def run_ours(args):
                     clocks=dict(sm_mhz=clocks.get("sm_mhz"), sm_max_mhz=clocks.get("sm_max_mhz"),
                                 reasons=clocks.get("reasons", []), samples=clocks.get("samples", 0),
                                 power_w_max=clocks.get("power_w_max")),
-                    e2e=e2e, gpu_launches=launches, roofline=roof, cpu_baseline=cpu, status=status)
+                    e2e=e2e, gpu_launches=launches, roofline=roof, cpu_baseline=cpu, parity=parity, status=status)
         print(json.dumps(line))
     ctx.close()
     if world > 1:
