@@ -78,11 +78,7 @@ static inline cudaError_t pvf_launch(void (*kernel)(KArgs...), dim3 grid, dim3 b
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-#ifdef PVF_NO_PDL
-    cfg.numAttrs = 0;
-#else
     cfg.numAttrs = 1;
-#endif
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -104,11 +100,7 @@ static inline cudaError_t pvf_launch_cluster2(void (*kernel)(KArgs...), dim3 gri
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-#ifdef PVF_NO_PDL
-    cfg.numAttrs = 1;
-#else
     cfg.numAttrs = 2;
-#endif
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif
