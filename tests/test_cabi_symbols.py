@@ -51,3 +51,28 @@ def test_error_strings_and_host_side_argument_checks():
     assert lib.pvf_score(None, None, 4, None, None, None, None, None) == binding.PVF_ERR_INVALID
     assert lib.pvf_workspace_bytes(None) == 0
     assert lib.pvf_create(None, None, None, None, 0, None, 0) == binding.PVF_ERR_INVALID
+
+
+def test_host_only_entry_points_work_without_a_gpu():
+    lib = binding.load()
+    # every error code has a message of its own
+    codes = [0, -1, -2, -3, -4, -5, -6, -7]
+    msgs = [binding.strerror(c) for c in codes]
+    assert len(set(msgs)) == len(codes) and binding.strerror(-99) == "unknown error"
+    # staging and bounce sizes are pure arithmetic on the shape
+    small = binding.pvf_shape(4096, 256, 64, 4, 4)
+    big = binding.pvf_shape(4096, 256, 128, 4, 4)
+    s_small = lib.pvf_host_staging_bytes(ctypes.byref(small))
+    s_big = lib.pvf_host_staging_bytes(ctypes.byref(big))
+    assert s_small >= 64 * 256 * 2 and s_big - s_small >= 64 * 256 * 2
+    b_small = lib.pvf_host_bounce_bytes(ctypes.byref(small))
+    assert 0 < b_small < s_small and s_small - b_small >= 64 * 256 * 2          # the bounce buffer holds no hidden states
+    bad = binding.pvf_shape(0, 256, 64, 4, 4)
+    assert lib.pvf_host_staging_bytes(ctypes.byref(bad)) == 0 and lib.pvf_host_bounce_bytes(ctypes.byref(bad)) == 0
+    # calls that need a context refuse a missing one instead of touching the device
+    assert lib.pvf_score(None, None, 4, None, None, None, None, None) == binding.PVF_ERR_INVALID
+    assert lib.pvf_attach_host_staging(None, None, 0) == binding.PVF_ERR_INVALID
+    assert lib.pvf_working_set(None, None, 1, 8, 4, 0, 0, None, None, None, None, None, 8, None) == binding.PVF_ERR_INVALID
+    assert lib.pvf_score_kernel_name(None, 4) is None
+    st = ctypes.c_int32(7)
+    assert lib.pvf_last_status(None, ctypes.byref(st)) == binding.PVF_ERR_INVALID
