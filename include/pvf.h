@@ -10,6 +10,15 @@
  *   pvf_select_drafts  planning candidates P_t^plan -> top-K drafts, else the AR fallback list
  *   pvf_verify         impact-set acceptance A_t^j, branch choice by C_total, AR k*, final commit
  *
+ * and, around the step:
+ *
+ *   pvf_working_set        rows of the next step from the canvas (block order, early cross-block revelation)
+ *   pvf_explore_commit     the appendix's Random / Planning exploration variants
+ *   pvf_calib_accumulate, pvf_calib_filter, pvf_set_plan_bitmap
+ *                          offline construction of the planning-token vocabulary
+ *   pvf_draft_step_host, pvf_verify_step_host      the step with host buffers
+ *   pvf_score_static       scoring without a context, for callers that must not allocate
+ *
  * Conventions common to all calls
  *   - Every data pointer is a DEVICE pointer owned by the caller unless it is marked "host".  The
  *     library never frees caller memory and keeps no pointer beyond a call, except the LM-head
