@@ -14,9 +14,10 @@
 // accumulators alternate, so the epilogue of one vocabulary tile overlaps the MMAs of the next.
 //
 // The GEMM kernel is a template over its tile shape (GemmCfg): vocabulary entries per accumulator,
-// 64-element k-panels per pipeline stage, stages; it serves 33 .. 128 rows.  More rows take the paired
-// kernel (pvf_score_gemm_pair_kernel: two blocks per 256-row tile, tcgen05 cta_group::2, each loading
-// half of every W tile).  Calls with at most 32 rows take a kernel with the operands swapped
+// 64-element k-panels per pipeline stage, stages; it serves 33 .. 128 rows and more than 8192 rows.
+// 129 .. 8192 rows take the paired kernel (pvf_score_gemm_pair_kernel: two blocks per 256-row tile,
+// tcgen05 cta_group::2, each loading half of every W tile) where the cost model prefers it.  Calls
+// with at most 32 rows take a kernel with the operands swapped
 // (pvf_score_stream_kernel): vocabulary on the lanes, rows on the columns, so that no tensor work is
 // spent on padding rows.
 //
