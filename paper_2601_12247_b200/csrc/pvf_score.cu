@@ -287,10 +287,14 @@ struct TileSplit {
     }
 };
 
-// Running softmax state of one row over the columns seen so far.
+// Running softmax state of one row over the columns seen so far.  The term of the maximum itself (e^0 = 1) is
+// kept OUT of the sum: beside it, the other terms of a peaked row (e^-17 = 4e-8 each, a hundred thousand of them,
+// half a per cent of the mass together) lie below the fp32 rounding unit of 1.0 and would be rounded away one by
+// one.  The row's normaliser is 1 + s.  The state is empty while arg is kNoArg.
+constexpr int kNoArg = 0x7fffffff;
 struct RowState {
     float m;      // running max
-    float s;      // sum e^{x - m}
+    float s;      // sum of e^{x - m} over every column except the one that holds the max
     float t;      // sum (x - m) e^{x - m}
     int arg;      // lowest id attaining m
 };
@@ -306,26 +310,33 @@ __device__ __forceinline__ void fold16(RowState &st, const uint32_t (&raw)[16], 
     float cm = x[0];
 #pragma unroll
     for (int i = 1; i < 16; ++i) cm = fmaxf(cm, x[i]);
+    int skip = -1;                                     // the column that becomes the new max: not a term of s
     if (cm > st.m) {                                   // strict: an equal later logit keeps the lower id
         int idx = 15;
 #pragma unroll
         for (int i = 14; i >= 0; --i) idx = (x[i] == cm) ? i : idx;
-        const float d = st.m - cm;                     // -inf on the first fold: the state is empty then
-        const float c = (st.s > 0.f) ? fast_exp2(d * kLog2e) : 0.f;
-        st.t = (st.s > 0.f) ? (st.t + d * st.s) * c : 0.f;
-        st.s *= c;
+        if (st.arg != kNoArg) {                        // the old max turns into an ordinary term
+            const float d = st.m - cm;
+            const float c = fast_exp2(d * kLog2e);
+            const float total = st.s + 1.f;
+            st.t = (st.t + d * total) * c;
+            st.s = total * c;
+        }
         st.m = cm;
         st.arg = col0 + idx;
+        skip = idx;
     }
+    float group = 0.f;                                 // the group's small terms are added up among themselves first
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
         if (kFull || i < n) {
             const float d = x[i] - st.m;
             const float e = fast_exp2(d * kLog2e);
-            st.s += e;
+            group += (i == skip) ? 0.f : e;
             st.t = fmaf(d, e, st.t);
         }
     }
+    st.s += group;
 }
 
 // One W tile of `tun` granules starting at granule tu0, columns x .. x+63, into b_dst.
@@ -483,7 +494,7 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
             const int row = m_tile * kTileM + row_in_tile;
             const bool warp_has_rows = m_tile * kTileM + quad * 32 < args.M;
             RowState st;
-            st.m = -INFINITY; st.s = 0.f; st.t = 0.f; st.arg = 0x7fffffff;
+            st.m = -INFINITY; st.s = 0.f; st.t = 0.f; st.arg = kNoArg;
             for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
                 int tu0, tun;
                 split.tile(tile, &tu0, &tun);
@@ -722,7 +733,7 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             const int row = row_base + row_in_tile;
             const bool warp_has_rows = row_base + quad * 32 < args.M;
             RowState st;
-            st.m = -INFINITY; st.s = 0.f; st.t = 0.f; st.arg = 0x7fffffff;
+            st.m = -INFINITY; st.s = 0.f; st.t = 0.f; st.arg = kNoArg;
             for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
                 int tu0, tun;
                 split.tile(tile, &tu0, &tun);
@@ -787,39 +798,51 @@ static_assert(kStreamStages >= 2 && kStreamStages <= kMaxStages && kStreamSmemBy
 // the end-of-block fold reuses the tile ring: 128 lanes x 32 rows x 16 bytes
 static_assert(kStreamStages * kStreamStageBytes >= kTileM * kStreamRows * 16, "fold scratch");
 
-// State (m, s, t, arg) absorbs one more logit x of vocabulary id v.
+// State (m, s, t, arg) absorbs one more logit x of vocabulary id v (s leaves out the max's own term, see RowState).
 __device__ __forceinline__ void state_push(float &m, float &s, float &t, int &arg, float x, int v)
 {
     constexpr float kLog2e = 1.4426950408889634f;
     if (x > m) {                                        // strict: ids ascend, so the lowest id keeps a tie
-        const float d = m - x;
-        const float c = (s > 0.f) ? fast_exp2(d * kLog2e) : 0.f;
-        t = (s > 0.f) ? (t + d * s) * c : 0.f;
-        s *= c;
+        if (arg != kNoArg) {
+            const float d = m - x;
+            const float c = fast_exp2(d * kLog2e);
+            const float total = s + 1.f;
+            t = (t + d * total) * c;
+            s = total * c;
+        }
         m = x;
         arg = v;
+    } else {
+        const float d = x - m;
+        const float e = fast_exp2(d * kLog2e);
+        s += e;
+        t = fmaf(d, e, t);
     }
-    const float d = x - m;
-    const float e = fast_exp2(d * kLog2e);
-    s += e;
-    t = fmaf(d, e, t);
 }
 
-// a <- a merged with b (two states over disjoint vocabulary sets).
+// a <- a merged with b (two states over disjoint vocabulary sets).  The larger max stays outside the sum; the
+// other state's max joins it as an ordinary term.
 __device__ __forceinline__ void state_merge(float4 &a, const float4 b)
 {
     constexpr float kLog2e = 1.4426950408889634f;
-    if (!(b.y > 0.f)) return;
-    if (!(a.y > 0.f)) { a = b; return; }
     const int ia = __float_as_int(a.w), ib = __float_as_int(b.w);
-    const float m = fmaxf(a.x, b.x);
-    const float da = a.x - m, db = b.x - m;
-    const float ca = fast_exp2(da * kLog2e), cb = fast_exp2(db * kLog2e);
-    const int arg = (a.x > b.x) ? ia : ((b.x > a.x) ? ib : min(ia, ib));
-    a.z = (a.z + da * a.y) * ca + (b.z + db * b.y) * cb;
-    a.y = a.y * ca + b.y * cb;
-    a.x = m;
-    a.w = __int_as_float(arg);
+    if (ib == kNoArg) return;
+    if (ia == kNoArg) { a = b; return; }
+    if (a.x > b.x || (a.x == b.x && ia < ib)) {
+        const float d = b.x - a.x;                      // <= 0
+        const float c = fast_exp2(d * kLog2e);
+        const float total = b.y + 1.f;
+        a.y += total * c;
+        a.z += (b.z + d * total) * c;
+    } else {
+        const float d = a.x - b.x;
+        const float c = fast_exp2(d * kLog2e);
+        const float total = a.y + 1.f;
+        a.y = b.y + total * c;
+        a.z = b.z + (a.z + d * total) * c;
+        a.x = b.x;
+        a.w = b.w;
+    }
 }
 
 __global__ void __launch_bounds__(kStreamThreads, 1)
@@ -945,7 +968,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
         float sm[kStreamRows], ss[kStreamRows], st[kStreamRows];
         int sa[kStreamRows];
 #pragma unroll
-        for (int i = 0; i < kStreamRows; ++i) { sm[i] = -INFINITY; ss[i] = 0.f; st[i] = 0.f; sa[i] = 0x7fffffff; }
+        for (int i = 0; i < kStreamRows; ++i) { sm[i] = -INFINITY; ss[i] = 0.f; st[i] = 0.f; sa[i] = kNoArg; }
         bool alive = true;
         for (int tile = 0; tile < n_tiles && alive; ++tile) {
             int tu0, tun;
@@ -991,7 +1014,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
             const float4 *scratch = reinterpret_cast<const float4 *>(tiles_ptr);
             const int e = threadIdx.x - 64;                              // 0..127
             const int row = e >> 2, part = e & 3;
-            float4 acc = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(0x7fffffff));
+            float4 acc = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(kNoArg));
             for (int l = 0; l < 32; ++l) state_merge(acc, scratch[row * kTileM + part * 32 + l]);
             for (int o = 1; o < 4; o <<= 1) {
                 float4 other;
@@ -1030,26 +1053,27 @@ pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int splits, i
     const float4 *p = partials + (size_t)row * splits;
     // lane-local pass: only the max and its lowest id
     float m = -INFINITY;
-    int arg = 0x7fffffff;
+    int arg = kNoArg;
     for (int i = lane; i < splits; i += 32) {
         const float4 v = p[i];
         const int a = __float_as_int(v.w);
-        if (v.y > 0.f && (v.x > m || (v.x == m && a < arg))) { m = v.x; arg = a; }
+        if (a != kNoArg && (v.x > m || (v.x == m && a < arg))) { m = v.x; arg = a; }
     }
     for (int o = 16; o > 0; o >>= 1) {
         const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
         const int a2 = __shfl_xor_sync(0xffffffffu, arg, o);
         if (m2 > m || (m2 == m && a2 < arg)) { m = m2; arg = a2; }
     }
-    // rescale every partial to the global max and add
+    // rescale every partial to the global max and add; a partial's sum leaves out its own max's term (1)
     double s = 0.0, t = 0.0;
     for (int i = lane; i < splits; i += 32) {
         const float4 v = p[i];
-        if (v.y > 0.f) {
+        if (__float_as_int(v.w) != kNoArg) {
             const double d = (double)v.x - (double)m;
             const double c = exp(d);
-            s += (double)v.y * c;
-            t += ((double)v.z + d * (double)v.y) * c;
+            const double total = 1.0 + (double)v.y;
+            s += total * c;
+            t += ((double)v.z + d * total) * c;
         }
     }
     for (int o = 16; o > 0; o >>= 1) {

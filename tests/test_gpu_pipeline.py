@@ -159,12 +159,24 @@ def test_config1b_sampled(llada):
     sampled_parity(ctx, st, w_bits, plan, np.array([0, 31, 32, 127, 128, 129, 200, 255]))
 
 
+def test_config2_full_step_on_the_oracles_own_scores(llada):
+    # every draft and verification row of config 2 scored by the oracle itself: decisions compared end to end
+    w_bits, _, _ = llada
+    st = synth.config2(w_bits=w_bits)
+    ctx = make_ctx(w_bits, st.plan_ids, 8192, 64, 16)          # config 2 has a planning vocabulary of its own
+    over, n_checked = verify_pass(ctx, st, *full_step(ctx, st))
+    assert n_checked >= st.n_seq // 2
+    ctx.close()
+
+
 def test_config2_sampled_rows_and_decisions_on_gpu_scores(llada):
     w_bits, plan, ctx = llada
     st = synth.config2(w_bits=w_bits)
     M = st.n_rows
     got = sampled_parity(ctx, st, w_bits, plan, np.unique(np.linspace(0, M - 1, 12).astype(int)))
-    # decisions are integer work: on the GPU's own fp32 scores they must equal the oracle's exactly
+    # consistency of the decision kernels with the scoring kernel's outputs: fed the same fp32 numbers, the
+    # oracle's decision rules must give the same sets (the scores themselves are checked on sampled rows above
+    # and on every row in test_config2_full_step_on_the_oracles_own_scores)
     p = st.params
     prm = params_of(st)
     seg, pos, act = t_i32(st.seg_off), t_i32(st.row_pos), t_u8(st.active)
@@ -243,3 +255,19 @@ def test_config3_large_batch_sampled(llada):
     gs = to_np(sel)
     for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
         assert np.array_equal(gs[k], osel[k]), k
+    # one whole sequence end to end on the oracle's own scores (512 rows is what the oracle scores in seconds)
+    b = 41
+    r0, r1 = int(st.seg_off[b]), int(st.seg_off[b + 1])
+    osc = oscore.score(w_bits, st.h_bits[r0:r1], plan)
+    check_score(got, osc, st.vocab, plan, rows=np.arange(r0, r1))
+    one = np.array([0, r1 - r0], np.int32)
+    ocm1 = ostep.commit(osc["conf"], osc["tok"], one, st.row_pos[r0:r1], st.active[r0:r1], p["tau_high"])
+    osel1 = ostep.select_drafts(osc["conf"], osc["tok"], osc["in_plan"], ocm1["commit"], one, st.row_pos[r0:r1],
+                                st.active[r0:r1], p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], p["budget"])
+    taus = [p["tau_high"], p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"]]
+    if not ((osc["gap"] < NEAR_TIE) | fragile_rows(osc["conf"], taus)).any():
+        assert np.array_equal(to_np(cm)["commit"][r0:r1], ocm1["commit"])
+        want_rows = np.where(osel1["draft_rows"][0] >= 0, osel1["draft_rows"][0] + r0, -1)
+        assert np.array_equal(gs["draft_rows"][b], want_rows)
+        assert gs["route"][b] == osel1["route"][0] and gs["n_drafts"][b] == osel1["n_drafts"][0]
+        assert gs["rem_off"][b + 1] - gs["rem_off"][b] == osel1["rem_off"][1]

@@ -138,3 +138,33 @@ def test_non_finite_hidden_rows_stay_in_bounds_and_do_not_disturb_other_rows(M):
     want = oscore.score(st.w_bits, st.h_bits[good], st.plan_ids)
     check_score(got, want, V, st.plan_ids, rows=good)
     ctx.close()
+
+
+@pytest.mark.parametrize("copies", [1, 32, 256])
+def test_small_tail_terms_are_not_lost_beside_a_dominant_logit(copies):
+    # One logit 11 .. 20 above a narrow bulk (hidden size 1024: the other logits spread by 0.5 only): every other
+    # term e^{x - max} is near or below the fp32 rounding unit of 1.0, yet there are 70000 of them and together
+    # they hold up to a per cent of the probability mass.  A running sum that contains the dominant term's 1.0
+    # rounds them away -- the more, the longer the vocabulary range one block sweeps, i.e. the more rows the call
+    # has: 64 distinct rows are scored once (128-row kernel, 148 ranges), 32 times over (2048 rows, paired kernel)
+    # and 256 times over (16384 rows, few ranges per row tile).
+    V, D, M = 70000, 1024, 64
+    w = synth.make_w(21, V, D)
+    targets = (np.arange(M) * 331 + 7) % V
+    amps = np.linspace(18.0, 32.0, M)
+    keys = np.stack([np.zeros(M, np.int64), np.arange(M), np.zeros(M, np.int64)], axis=1)
+    h = synth.make_hidden_rows(w, targets, amps, 21, synth.TAG_NOISE, keys)
+    plan = synth.make_plan_ids(21, V, 64)
+    want = oscore.score(w, h, plan)
+    assert ((1.0 - want["conf"]) > 1e-3).sum() >= M // 4 and want["gap"].min() > 8.0     # the case under test is present
+    ctx = make_ctx(w, plan, M * copies)
+    got = to_np(ctx.score(upload_bits(np.tile(h, (copies, 1)))))
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    for c in sorted({0, copies // 2, copies - 1}):
+        rows = np.arange(c * M, (c + 1) * M)
+        check_score(got, want, V, plan, rows=rows)
+        # far inside the tolerance: a lost tail shows as an error of a fifth to a half of 1 - conf (up to 1e-3 here)
+        assert np.max(np.abs(got["conf"][rows] - want["conf"])) <= 1e-4
+        assert np.max(np.abs(got["ent"][rows] - want["ent"])) <= 3e-4
+    ctx.close()
