@@ -255,6 +255,27 @@ def test_config3_large_batch_sampled(llada):
     gs = to_np(sel)
     for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
         assert np.array_equal(gs[k], osel[k]), k
+    # every one of the 32768 rows against a second reference: torch's fp64 matmul and log-softmax on the GPU (not
+    # the oracle -- the oracle checks 8 + 512 rows of this launch above and below, and pins this reference on the
+    # sampled rows); it is what catches an error that only a few rows in ten thousand show
+    wd = ctx.w_head.double()
+    hd = upload_bits(st.h_bits)
+    ref_conf = np.empty(st.n_rows); ref_ent = np.empty(st.n_rows); ref_tok = np.empty(st.n_rows, np.int64); ref_gap = np.empty(st.n_rows)
+    for r0 in range(0, st.n_rows, 1024):
+        lp = torch.log_softmax(hd[r0:r0 + 1024].double() @ wd.t(), dim=1)
+        top2 = lp.topk(2, dim=1)
+        ref_conf[r0:r0 + 1024] = top2.values[:, 0].exp().cpu().numpy()
+        ref_tok[r0:r0 + 1024] = top2.indices[:, 0].cpu().numpy()
+        ref_gap[r0:r0 + 1024] = (top2.values[:, 0] - top2.values[:, 1]).cpu().numpy()
+        ref_ent[r0:r0 + 1024] = (-(lp.exp() * lp).sum(dim=1)).cpu().numpy()
+        del lp
+    want_s = oscore.score(w_bits, st.h_bits[sample], plan)
+    assert np.max(np.abs(ref_conf[sample] - want_s["conf"])) < 1e-9 and np.max(np.abs(ref_ent[sample] - want_s["ent"])) < 1e-9
+    assert np.array_equal(ref_tok[sample], want_s["tok"])
+    assert np.max(np.abs(got["conf"] - ref_conf)) <= 1e-3 and np.max(np.abs(got["ent"] - ref_ent)) <= 1e-3
+    clear = ref_gap >= NEAR_TIE
+    assert np.array_equal(got["tok"][clear], ref_tok[clear]) and (~clear).sum() < 100
+    del wd
     # one whole sequence end to end on the oracle's own scores (512 rows is what the oracle scores in seconds)
     b = 41
     r0, r1 = int(st.seg_off[b]), int(st.seg_off[b + 1])
