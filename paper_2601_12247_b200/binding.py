@@ -56,6 +56,15 @@ def load() -> ctypes.CDLL:
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
+            # not built yet: build it now if this machine has nvcc; there is no CPU or PyTorch fallback
+            try:
+                from . import build as _build
+                if os.path.abspath(LIB_PATH) == os.path.abspath(_build.LIB):
+                    _build.build()
+            except Exception as exc:
+                raise RuntimeError("libpvf.so is not built and could not be built here (%s): run "
+                                   "`python -m paper_2601_12247_b200.build` (there is no CPU or PyTorch fallback)" % exc)
+        if not os.path.exists(LIB_PATH):
             raise RuntimeError("libpvf.so is not built: run `python -m paper_2601_12247_b200.build` "
                                "(there is no CPU or PyTorch fallback)")
         lib = ctypes.CDLL(LIB_PATH)
