@@ -233,9 +233,13 @@ def run_ours(args):
     o_ver = dict(accept=torch.empty((st.n_seq, K), dtype=torch.uint8, device=dev),
                  choice=torch.empty(st.n_seq, dtype=torch.int32, device=dev),
                  final_commit=torch.empty(M, dtype=torch.uint8, device=dev))
+    # The projection kernel is timed on every `event_every`-th step of the timed region: events around a launch
+    # cost the overlap of its set-up with the previous kernel, so timing all of them would slow the step it measures.
+    event_every = 8 if args.steps >= 64 else 1
+    n_event_steps = (args.steps + event_every - 1) // event_every
     ev_pairs = []
     ev_pool = []
-    for _ in range(2 * args.steps):                # created (and first recorded) outside the timed region
+    for _ in range(2 * n_event_steps):             # created (and first recorded) outside the timed region
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(); b.record()
         ev_pool.append((a, b))
@@ -243,6 +247,8 @@ def run_ours(args):
 
     def step(h_dev, hv_dev, timed_events=False):
         launches = 0
+        if not timed_events:
+            ctx.set_score_events(None, None)
         if timed_events:
             a, b = ev_pool.pop()
             ctx.set_score_events(a, b); ev_pairs.append((a, b, M))
@@ -278,8 +284,8 @@ def run_ours(args):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches = 0
     e0.record()
-    for _ in range(args.steps):
-        launches += step(h, hv, timed_events=True)
+    for i in range(args.steps):
+        launches += step(h, hv, timed_events=(i % event_every == 0))
     e1.record()
     barrier()
     clocks = sampler.stop()
@@ -339,7 +345,7 @@ def run_ours(args):
         traffic = NCU_TRAFFIC_PAIR_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
     else:
         traffic = None
-    roof.update(traffic=traffic, kernel="+".join(kernels), launches=n_gemm, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
+    roof.update(traffic=traffic, kernel="+".join(kernels), launches=n_gemm, timed_every_nth_step=event_every, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
                 algorithmic_bytes_per_launch=alg_bytes / max(n_gemm, 1), peak_source=peaks["source"] +
                 (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy bandwidth)"))
 
