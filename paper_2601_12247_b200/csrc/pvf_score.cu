@@ -795,6 +795,7 @@ constexpr int kStreamSecondIssuerWarp = 6;
 constexpr int kStreamThreads = 224;                                 // producer, issuer, 4 epilogue warps, issuer
 constexpr int kStreamSmemBytes = kStreamStages * kStreamStageBytes + 1024 + kStreamControlBytes;
 static_assert(kStreamStages >= 2 && kStreamStages <= kMaxStages && kStreamSmemBytes <= 227 * 1024, "streaming ring");
+static_assert(kStreamTileN == 2 * kTileM, "each of the two MMA slices reads kTileM W rows of the stage");
 // the end-of-block fold reuses the tile ring: 128 lanes x 32 rows x 16 bytes
 static_assert(kStreamStages * kStreamStageBytes >= kTileM * kStreamRows * 16, "fold scratch");
 
