@@ -38,9 +38,9 @@ UNIT = "positions/s"
 # the ncu captures summarised under profiles/ (None = not captured since the kernel last changed).  The
 # streaming kernel's config-1a launch is captured as is; launches of the GEMM kernel scale the captured
 # per-pass traffic by their number of passes over W ("waves").
-NCU_TRAFFIC_STREAM_LAUNCH = 1.04074e9
-NCU_TRAFFIC_GEMM_PER_WAVE = 1.162e9
-NCU_TRAFFIC_PAIR_PER_WAVE = 1.0497e9
+NCU_TRAFFIC_STREAM_LAUNCH = 1.04217e9
+NCU_TRAFFIC_GEMM_PER_WAVE = 1.277e9
+NCU_TRAFFIC_PAIR_PER_WAVE = 1.0490e9
 
 
 def load_peaks():
