@@ -51,6 +51,11 @@ struct pvf_score_geometry {
     int streaming;   // 1: at most 32 rows, handled by the swapped-operand streaming kernel
     int paired;      // 1: more than 128 rows, handled by the paired (cta_group::2) kernel; then m_tiles counts
                      //    256-row tiles, units granules of 32 entries, mb / splits pairs of blocks
+    int swapped;     // 1: handled by the swapped paired kernel; m_tiles counts row tiles of n_pad rows, units
+                     //    granules of 32 entries, mb / splits pairs of blocks
+    int n_pad;       // swapped: rows per row tile (multiple of 32, at most 256)
+    int stages;      // swapped: pipeline stages that fit the shared-memory ring
+    int parts;       // partial states per row handed to the merge kernel (splits, or 2 * splits when swapped)
 };
 pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm);
 size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm);

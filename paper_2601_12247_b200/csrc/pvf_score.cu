@@ -19,7 +19,8 @@
 // tcgen05 cta_group::2, each loading half of every W tile) where the cost model prefers it.  Calls
 // with at most 32 rows take a kernel with the operands swapped
 // (pvf_score_stream_kernel): vocabulary on the lanes, rows on the columns, so that no tensor work is
-// spent on padding rows.
+// spent on padding rows.  33 .. 64 and 129 .. 192 rows, where 128- and 256-row tiles would be mostly
+// padding, take the paired kernel with swapped operands (pvf_score_swap_pair_kernel).
 //
 // Work split.  Rows form tiles of 128, the vocabulary granules of 16 entries.  `mb` row tiles are
 // in flight at once, each swept by `splits` blocks over disjoint vocabulary ranges (mb * splits
@@ -51,6 +52,12 @@
 #endif
 #ifndef PVF_PAIR_MAX_ROWS
 #define PVF_PAIR_MAX_ROWS 8192   // rows up to which the paired kernel is considered
+#endif
+#ifndef PVF_SWAP_SMALL_MAX_ROWS
+#define PVF_SWAP_SMALL_MAX_ROWS 64     // 33 .. this many rows take the swapped paired kernel
+#endif
+#ifndef PVF_SWAP_RAGGED_MAX_ROWS
+#define PVF_SWAP_RAGGED_MAX_ROWS 192   // and so do 129 .. this many rows (at most 256)
 #endif
 
 namespace {
@@ -112,7 +119,9 @@ struct ScoreArgs {
     int units;           // ceil(V / 16)
     int m_tiles, mb, splits, waves;
     int a_rows;          // rows per H box
-    float4 *partials;    // [M][splits]
+    int n_pad, stages;   // swapped paired kernel: rows per row tile (MMA N), pipeline stages
+    int parts;           // partial states per row (row stride of `partials`)
+    float4 *partials;    // [M][parts]
     int32_t *status;
 };
 
@@ -1038,6 +1047,231 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     }
 }
 
+// ---------------------------------------------------------------------------------- swapped paired kernel
+// 33 .. 256 rows in one row tile: the launch sits at the ridge, where HBM, the tensor pipe and the power cap all
+// matter, and 128- or 256-row MMAs over a ragged row count waste tensor work (and with it clock).  Here the
+// operands of the paired kernel change places: the two blocks of a pair hold 2 x 128 vocabulary entries on
+// their accumulator lanes (each loads its own 128-entry W tile, so W still crosses L2 -> SM once) and the
+// scored rows are the N columns, N = the row tile padded to 32 (each block loads half of the H tile):
+//     D[v][m] = sum_k W[v][k] * H[m][k],   one 256 x N x 16 MMA (cta_group::2) per 16 elements of k.
+// At most 31 padded rows are wasted.  Measured against the other two kernels (each alone for seconds, so that
+// the power cap has settled, and in short bursts) it wins where they pad most: 33 .. 64 rows (4 .. 5 %) and
+// 129 .. 192 rows (4 .. 9 %); with full 128- or 256-row tiles they are 3 .. 9 % faster, so the geometry picks it
+// for those two windows only.
+//
+// Epilogue: a warp owns 32 vocabulary lanes and reads 32 rows (columns) at a time.  It turns that 32 x 32 block
+// around through a padded shared-memory tile of its own, after which lane i holds row i's 32 logits and folds
+// them into the running state of row chunk*32 + i exactly as the GEMM kernels' epilogue does (no warp-wide
+// reductions: those serialise on their latency with one epilogue warp per scheduler).  At the end of the block's
+// range the four warps' states fold through the same shared memory and the block writes one partial state per
+// row: 2 x splits partial states per row reach the merge kernel.
+//
+// The ring has as many stages as fit: a stage is the block's 16 KiB W tile plus its half of the H tile.
+constexpr int kSwapWBytes = kTileM * kRowBytes;                      // 16 KiB
+constexpr int kSwapMaxRowsPerTile = 256;                             // MMA N limit
+constexpr int kSwapTmemCols = 512;                                   // 2 accumulators x 256 columns
+constexpr int kSwapTurnPitch = 36;                                   // words per lane of a warp's 32 x 32 fp32 block: 16-byte
+                                                                     // aligned rows, conflict-free 128-bit stores and column reads
+constexpr int kSwapWarpScratchBytes = 32 * kSwapTurnPitch * 4;       // that block; later the warp's 256 row states (4 KiB) for the fold
+constexpr int kSwapScratchBytes = 4 * kSwapWarpScratchBytes;
+static_assert(kSwapWarpScratchBytes >= kSwapMaxRowsPerTile * 16 && kSwapWarpScratchBytes % 16 == 0, "fold scratch");
+constexpr int kSwapRingBytes = 204 * 1024;
+constexpr int kSwapMaxStages = 12;
+constexpr int kSwapSmemBytes = kSwapRingBytes + 1024 + 512 + kSwapScratchBytes;
+static_assert(kSwapSmemBytes <= 227 * 1024, "swapped ring");
+static_assert(kSwapMaxStages <= kMaxStages, "barrier arrays");
+static_assert(PVF_SWAP_SMALL_MAX_ROWS <= kSwapMaxRowsPerTile && PVF_SWAP_RAGGED_MAX_ROWS <= kSwapMaxRowsPerTile, "one row tile");
+
+__global__ void __launch_bounds__(kThreads, 1)
+pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ WMaps tm_w, const ScoreArgs args)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
+    uint8_t *tiles_ptr = smem_raw + (tiles_addr - raw_addr);
+    const int n_pad = args.n_pad;                                        // rows per row tile = MMA N (multiple of 32)
+    const int n_stages = args.stages;
+    const uint32_t h_bytes = (uint32_t)(n_pad / 2) * kRowBytes;          // this block's half of the H tile
+    const uint32_t stage_bytes = (uint32_t)kSwapWBytes + h_bytes;
+    SharedControl *ctl = reinterpret_cast<SharedControl *>(tiles_ptr + (size_t)n_stages * stage_bytes);
+    uint8_t *scratch = reinterpret_cast<uint8_t *>(ctl) + 512;          // one kSwapWarpScratchBytes region per epilogue warp
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();                            // 0: even block (issues the MMAs), 1: its peer
+    const int q = blockIdx.x >> 1;                                       // the pair's vocabulary range
+    int u0, u1;
+    split_range(args.units, args.splits, q, &u0, &u1);                   // granules of 32 entries
+    const TileSplit split(u0, u1, kPairUnitsPerTile);
+    const int n_tiles = split.n_tiles;
+    const int k_steps = args.num_kb;
+
+    if (threadIdx.x == 0) init_pipeline_barriers(ctl, n_stages, 1, 2 * kEpilogueThreads);
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.size[kPairUnitsPerTile - 1]) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctl->tmem_base)), "r"(kSwapTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = ctl->tmem_base;
+    pvf_grid_dependency_wait();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (one per block)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool alive = true;
+            const int row0 = (int)rank * (n_pad / 2);                               // this block's half of the rows
+            for (int tile = 0; tile < n_tiles && alive; ++tile) {
+                int tu0, tun;
+                split.tile(tile, &tu0, &tun);
+                const uint32_t bytes = 2u * ((uint32_t)tun * kUnitBytes + h_bytes);                     // both blocks
+                const int w_row = tu0 * kPairUnit + (int)rank * tun * kUnit;                            // this block's entries
+                for (int step = 0; step < k_steps; ++step) {
+                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                    const uint32_t full = smem_u32(&ctl->full[stage]);
+                    const uint32_t w_dst = tiles_addr + (uint32_t)stage * stage_bytes;
+                    if (rank == 0) mbar_arrive_expect_tx(full, bytes);
+                    tma_load_2d_pair(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
+                    tma_load_2d_pair(w_dst + kSwapWBytes, &tm_h, full, step * kBlockK, row0);
+                    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!alive) {
+                const unsigned long long t0 = global_timer_ns();
+                while (global_timer_ns() - t0 < 200000ull) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (even block only)
+        if (lane == 0 && rank == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool alive = true;
+            const uint32_t idesc = instr_desc_bf16_m256(n_pad);
+            for (int tile = 0; tile < n_tiles && alive; ++tile) {
+                const uint32_t buf = (uint32_t)tile & 1u;
+                const uint32_t acc_phase = ((uint32_t)tile >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), acc_phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                tc_fence_after_sync();
+                const uint32_t tmem_d = tmem_base + buf * kSwapMaxRowsPerTile;
+                for (int step = 0; step < k_steps; ++step) {
+                    if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, ctl, args.status)) { alive = false; break; }
+                    tc_fence_after_sync();
+                    // A ragged vocabulary tile leaves stale bytes on the W tile's last rows: lanes the epilogue skips.
+                    const uint32_t w_addr = tiles_addr + (uint32_t)stage * stage_bytes;
+                    const uint64_t w_desc = smem_desc_k_major_sw128(w_addr);
+                    const uint64_t h_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / 16; ++k)
+                        tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h_desc + (uint64_t)(k * 2), idesc,
+                                         (step | k) != 0 ? 1u : 0u);
+                    tc_commit_pair(smem_u32(&ctl->empty[stage]));
+                    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
+                }
+                if (alive) tc_commit_pair(smem_u32(&ctl->acc_full[buf]));
+            }
+            if (!alive) {
+                tc_commit_pair_local(smem_u32(&ctl->drain));
+                const unsigned long long t0 = global_timer_ns();
+                while (!mbar_try_wait(smem_u32(&ctl->drain), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax epilogue (both blocks)
+        const int quad = warp & 3;                                       // tensor-memory lanes quad*32 .. quad*32+31
+        const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
+        const int n_chunks = n_pad >> 5;                                 // 32-row column groups
+        const int e_thread = quad * 32 + lane;
+        float *turn = reinterpret_cast<float *>(scratch + quad * kSwapWarpScratchBytes);          // [32 lanes][kSwapTurnPitch]
+        float4 *fold_mine = reinterpret_cast<float4 *>(scratch + quad * kSwapWarpScratchBytes);   // [256 rows], after the sweep
+        bool alive = true;
+        RowState st[kSwapMaxRowsPerTile / 32];                           // lane i: state of row chunk*32 + i
+#pragma unroll
+        for (int c = 0; c < kSwapMaxRowsPerTile / 32; ++c) { st[c].m = -INFINITY; st[c].s = 0.f; st[c].t = 0.f; st[c].arg = kNoArg; }
+        for (int tile = 0; tile < n_tiles && alive; ++tile) {
+            int tu0, tun;
+            split.tile(tile, &tu0, &tun);
+            const uint32_t buf = (uint32_t)tile & 1u;
+            const uint32_t acc_phase = ((uint32_t)tile >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), acc_phase, ctl, args.status)) { alive = false; break; }
+            tc_fence_after_sync();
+            const int block_v0 = tu0 * kPairUnit + (int)rank * tun * kUnit;         // vocabulary id on this block's lane 0
+            const int block_end = min(block_v0 + tun * kUnit, args.V);
+            const int warp_v0 = block_v0 + quad * 32;
+            const int n_real = min(32, block_end - warp_v0);                        // vocabulary entries on this warp's lanes
+            if (n_real > 0) {                                                        // warp-uniform
+#pragma unroll
+                for (int c = 0; c < kSwapMaxRowsPerTile / 32; ++c) {
+                    if (c < n_chunks) {                                              // block-uniform
+                        uint32_t lo[16], hi[16];
+                        const uint32_t col = lane_addr + buf * kSwapMaxRowsPerTile + c * 32;
+                        tmem_ld16(col, lo);
+                        tmem_ld16(col + 16, hi);
+                        tmem_ld_wait();
+                        uint4 *mine = reinterpret_cast<uint4 *>(turn + lane * kSwapTurnPitch);       // lane = vocabulary entry
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            mine[j] = make_uint4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
+                            mine[4 + j] = make_uint4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
+                        }
+                        __syncwarp();
+#pragma unroll
+                        for (int half = 0; half < 2; ++half) {                       // lane = row, 16 vocabulary entries at a time
+                            const int n = n_real - half * 16;
+                            if (n > 0) {
+                                uint32_t x[16];
+#pragma unroll
+                                for (int l = 0; l < 16; ++l) x[l] = __float_as_uint(turn[(half * 16 + l) * kSwapTurnPitch + lane]);
+                                if (n >= 16) fold16<true>(st[c], x, warp_v0 + half * 16, 16);
+                                else fold16<false>(st[c], x, warp_v0 + half * 16, n);
+                            }
+                        }
+                        __syncwarp();
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive_even_block(smem_u32(&ctl->acc_empty[buf]));
+        }
+        // Fold the block's four warps and write the block's partial state of every row.  Every epilogue thread
+        // reaches the barrier, aborting or not.
+        if (alive) {
+#pragma unroll
+            for (int c = 0; c < kSwapMaxRowsPerTile / 32; ++c)
+                if (c < n_chunks)
+                    fold_mine[c * 32 + lane] = make_float4(st[c].m, st[c].s, st[c].t, __int_as_float(st[c].arg));
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+        if (alive && !ctl->abort_flag) {
+            for (int row = e_thread; row < args.M; row += kEpilogueThreads) {
+                float4 acc = reinterpret_cast<const float4 *>(scratch)[row];
+#pragma unroll
+                for (int o = 1; o < 4; ++o)
+                    state_merge(acc, reinterpret_cast<const float4 *>(scratch + o * kSwapWarpScratchBytes)[row]);
+                args.partials[(size_t)row * args.parts + 2 * q + (int)rank] = acc;
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();
+    pvf_launch_dependents();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kSwapTmemCols) : "memory");
+    }
+}
+
 // ---------------------------------------------------------------------------------- merge kernel
 // One warp per row: combines the row's `splits` partial states (ascending vocabulary ranges) in
 // fp64 and writes token, confidence, entropy and planning-vocabulary membership.
@@ -1143,7 +1377,9 @@ int raise_shared_memory_limits()
         cudaFuncSetAttribute(pvf_score_gemm_kernel<GeneralCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              GeneralCfg::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(pvf_score_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kPairSmemBytes) != cudaSuccess)
+                             kPairSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(pvf_score_swap_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             kSwapSmemBytes) != cudaSuccess)
         return PVF_ERR_CUDA;
     return PVF_OK;
 }
@@ -1165,12 +1401,15 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
     a.units = g.units;
     a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
     a.a_rows = g.a_rows;
+    a.n_pad = g.n_pad; a.stages = g.stages; a.parts = g.parts;
     a.partials = partials;
     a.status = status;
     const bool timed = ev_start && ev_stop;
     if (timed && cudaEventRecord(ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
     cudaError_t e;
-    if (g.paired)
+    if (g.swapped)
+        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(kThreads), kSwapSmemBytes, s, tm_h, maps, a);
+    else if (g.paired)
         e = pvf_launch_cluster2(pvf_score_gemm_pair_kernel, dim3(g.ctas), dim3(kThreads), kPairSmemBytes, s, tm_h, maps, a);
     else if (g.streaming)
         e = pvf_launch(pvf_score_stream_kernel, dim3(g.ctas), dim3(kStreamThreads), kStreamSmemBytes, s, tm_h, maps, a);
@@ -1180,7 +1419,7 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
     if (timed && cudaEventRecord(ev_stop, s) != cudaSuccess) return PVF_ERR_CUDA;
     const int warps_per_block = 8;
     e = pvf_launch(pvf_score_merge_kernel, dim3((M + warps_per_block - 1) / warps_per_block), dim3(warps_per_block * 32), 0, s,
-                   (const float4 *)partials, M, g.splits, V, plan_bitmap, tok, conf, ent, in_plan);
+                   (const float4 *)partials, M, g.parts, V, plan_bitmap, tok, conf, ent, in_plan);
     return e == cudaSuccess ? PVF_OK : PVF_ERR_CUDA;
 }
 
@@ -1240,9 +1479,23 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm)
         const SplitPlan pp = plan_split(M, V, D, n_sm / 2, 2 * kTileM, kPairUnit, kMaxConcurrentTiles / 2);
         if (pp.waves > 0 && pp.cost <= 1.05 * p.cost) { p = pp; g.paired = 1; }
     }
+    g.swapped = 0; g.n_pad = 0; g.stages = 0;
+    if (n_sm >= 2 && ((M > kStreamRows && M <= PVF_SWAP_SMALL_MAX_ROWS) || (M > kTileM && M <= PVF_SWAP_RAGGED_MAX_ROWS))) {
+        // Swapped paired kernel: one row tile padded to a multiple of 32 rows (the MMA's N), every pair of SMs
+        // sweeps one vocabulary range.  Chosen where the other kernels would pad the rows most (see the kernel).
+        g.swapped = 1; g.paired = 0;
+        g.n_pad = ((M + 31) / 32) * 32;
+        g.a_rows = g.n_pad / 2;
+        const int stage_bytes = kSwapWBytes + (g.n_pad / 2) * kRowBytes;
+        g.stages = kSwapRingBytes / stage_bytes < kSwapMaxStages ? kSwapRingBytes / stage_bytes : kSwapMaxStages;
+        p.m_tiles = 1; p.mb = 1; p.waves = 1;
+        p.units = (V + kPairUnit - 1) / kPairUnit;
+        p.splits = n_sm / 2 < p.units ? n_sm / 2 : p.units;
+    }
     g.m_tiles = p.m_tiles; g.units = p.units;
     g.mb = p.mb; g.splits = p.splits; g.waves = p.waves;
-    g.ctas = g.mb * g.splits * (g.paired ? 2 : 1);
+    g.ctas = g.mb * g.splits * ((g.paired || g.swapped) ? 2 : 1);
+    g.parts = g.splits * (g.swapped ? 2 : 1);
     return g;
 }
 
@@ -1250,10 +1503,16 @@ size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm)
 {
     size_t worst = 0;
     const int max_tiles = (shape->max_rows + kTileM - 1) / kTileM;
-    for (int t = 1; t <= max_tiles; ++t) {                          // every 128-row step changes the geometry at most once
-        const int rows = t * kTileM < shape->max_rows ? t * kTileM : shape->max_rows;
+    // Within one kernel choice and row-tile count the need grows with the rows, so it peaks at the upper end of
+    // every 128-row step and of the swapped paired kernel's two windows.
+    for (int t = 1; t <= max_tiles + 2; ++t) {
+        int rows = t * kTileM;
+        if (t == max_tiles + 1) rows = PVF_SWAP_SMALL_MAX_ROWS;
+        if (t == max_tiles + 2) rows = PVF_SWAP_RAGGED_MAX_ROWS;
+        if (rows > shape->max_rows) rows = shape->max_rows;
+        if (rows <= 0) continue;
         const pvf_score_geometry g = pvf_score_geometry_for(rows, shape->vocab, shape->hidden, n_sm);
-        const size_t need = (size_t)rows * g.splits * sizeof(float4);
+        const size_t need = (size_t)rows * g.parts * sizeof(float4);
         worst = need > worst ? need : worst;
     }
     return worst;
@@ -1295,7 +1554,7 @@ int pvf_score_plan_for_shape(int32_t vocab, int32_t hidden, int32_t n_sm, int32_
     if (ctas) *ctas = g.ctas;
     if (splits) *splits = g.splits;
     if (waves) *waves = g.waves;
-    if (kernel) *kernel = g.streaming ? 0 : (g.paired ? 2 : 1);
+    if (kernel) *kernel = g.streaming ? 0 : (g.swapped ? 3 : (g.paired ? 2 : 1));
     if (row_tiles) *row_tiles = g.m_tiles;
     if (tiles_per_wave) *tiles_per_wave = g.mb;
     return PVF_OK;
@@ -1305,7 +1564,8 @@ const char *pvf_score_kernel_name(pvf_ctx *ctx, int32_t M)
 {
     if (!ctx || M <= 0 || M > ctx->shape.max_rows) return nullptr;
     const pvf_score_geometry g = pvf_score_geometry_for(M, ctx->shape.vocab, ctx->shape.hidden, ctx->n_sm);
-    return g.streaming ? "pvf_score_stream_kernel" : (g.paired ? "pvf_score_gemm_pair_kernel" : "pvf_score_gemm_kernel");
+    return g.streaming ? "pvf_score_stream_kernel"
+                       : (g.swapped ? "pvf_score_swap_pair_kernel" : (g.paired ? "pvf_score_gemm_pair_kernel" : "pvf_score_gemm_kernel"));
 }
 
 int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
@@ -1317,7 +1577,7 @@ int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
     if (((uintptr_t)hidden & 15) != 0) return PVF_ERR_ALIGN;
     const int V = ctx->shape.vocab, D = ctx->shape.hidden;
     const pvf_score_geometry g = pvf_score_geometry_for(M, V, D, ctx->n_sm);
-    if ((size_t)M * g.splits * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
+    if ((size_t)M * g.parts * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
     return launch_score(g, hidden, M, V, D, ctx->tm_w, ctx->partials, &ctx->words->status, ctx->plan_bitmap, tok, conf,
                         ent, in_plan, (cudaStream_t)stream, ctx->ev_start, ctx->ev_stop);
 }
@@ -1386,7 +1646,7 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     int rc = static_device_state(&st);
     if (rc != PVF_OK) return rc;
     const pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden_size, st->n_sm);
-    if ((size_t)M * g.splits * sizeof(float4) > kStaticPartialsBytes) return PVF_ERR_TOO_LARGE;
+    if ((size_t)M * g.parts * sizeof(float4) > kStaticPartialsBytes) return PVF_ERR_TOO_LARGE;
 
     CUtensorMap w_levels[kWBoxSizes];
     if ((rc = make_w_maps(w_levels, w_head, vocab, hidden_size)) != PVF_OK) return rc;

@@ -216,14 +216,16 @@ def test_paired_kernel_two_waves_sampled(llada):
 
 
 def test_second_model_shape_sampled():
-    # Dream-7B-like LM head: 56 k-panels, 9504 vocabulary granules (64.2 per block): all three kernels
+    # Dream-7B-like LM head: 56 k-panels, 9504 vocabulary granules (64.2 per block): all four kernels
     V, D = synth.DREAM_VOCAB, synth.DREAM_HIDDEN
     w_bits = synth.make_w(1005, V, D)
     plan = synth.make_plan_ids(1005, V, 2048)
     ctx = make_ctx(w_bits, plan, 512, 8, 8)
     st = synth.config1("b", stress=True, w_bits=w_bits, vocab=V, hidden=D)
     for rows, kernel, sample in ((32, "pvf_score_stream_kernel", np.array([0, 1, 15, 16, 30, 31])),
+                                 (48, "pvf_score_swap_pair_kernel", np.array([0, 23, 24, 32, 47])),
                                  (100, "pvf_score_gemm_kernel", np.array([0, 31, 32, 64, 99])),
+                                 (170, "pvf_score_swap_pair_kernel", np.array([0, 95, 96, 128, 169])),
                                  (256, "pvf_score_gemm_pair_kernel", np.array([0, 127, 128, 129, 255]))):
         assert ctx.score_kernel_name(rows) == kernel
         got = to_np(ctx.score(upload_bits(st.h_bits[:rows])))
