@@ -34,13 +34,16 @@ if ROOT not in sys.path:
 METRIC = "masked positions scored/s per fused PVF step"
 UNIT = "positions/s"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the projection kernel, from
-# the ncu captures summarised under profiles/ (None = not captured since the kernel last changed).  The
-# streaming kernel's config-1a launch is captured as is; launches of the GEMM kernel scale the captured
-# per-pass traffic by their number of passes over W ("waves").
-NCU_TRAFFIC_STREAM_LAUNCH = 1.04217e9
-NCU_TRAFFIC_GEMM_PER_WAVE = 1.277e9
-NCU_TRAFFIC_PAIR_PER_WAVE = 1.0490e9
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one pass over W ("wave") of each projection
+# kernel, from the ncu captures summarised under profiles/ (None = not captured since the kernel last changed).
+# The streaming and swapped paired kernels' launches are one pass; launches of the GEMM kernels scale the
+# captured per-pass traffic by their number of passes.
+NCU_TRAFFIC_PER_WAVE = {
+    "pvf_score_stream_kernel": 1.04217e9,
+    "pvf_score_gemm_kernel": 1.277e9,
+    "pvf_score_gemm_pair_kernel": 1.0490e9,
+    "pvf_score_swap_pair_kernel": 1.0495e9,
+}
 
 
 def load_peaks():
@@ -337,12 +340,9 @@ def run_ours(args):
         roof = dict(bound="tensor", achieved=alg_flops / t_gemm / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
     kernels = sorted({ctx.score_kernel_name(r) for _, _, r in ev_pairs})
-    if kernels == ["pvf_score_stream_kernel"]:
-        traffic = NCU_TRAFFIC_STREAM_LAUNCH
-    elif kernels == ["pvf_score_gemm_kernel"] and NCU_TRAFFIC_GEMM_PER_WAVE is not None:
-        traffic = NCU_TRAFFIC_GEMM_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
-    elif kernels == ["pvf_score_gemm_pair_kernel"] and NCU_TRAFFIC_PAIR_PER_WAVE is not None:
-        traffic = NCU_TRAFFIC_PAIR_PER_WAVE * sum(ctx.score_plan(r)["waves"] for _, _, r in ev_pairs) / max(n_gemm, 1)
+    per_launch = [NCU_TRAFFIC_PER_WAVE.get(ctx.score_kernel_name(r)) for _, _, r in ev_pairs]
+    if per_launch and all(t is not None for t in per_launch):       # average launch of the timed mix
+        traffic = sum(t * ctx.score_plan(r)["waves"] for t, (_, _, r) in zip(per_launch, ev_pairs)) / n_gemm
     else:
         traffic = None
     roof.update(traffic=traffic, kernel="+".join(kernels), launches=n_gemm, timed_every_nth_step=event_every, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
