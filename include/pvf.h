@@ -128,14 +128,14 @@ int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int3
 /* The same plan from shapes alone (no context, no device): n_sm = number of SMs to plan for.  `kernel` (may be
  * NULL) receives 0 for the streaming kernel, 1 for the 128-row GEMM kernel, 2 for the paired kernel, 3 for the paired
  * kernel with swapped operands; `row_tiles` the number of row tiles (256 rows in the paired kernel, one tile of up
- * to 256 rows in the swapped paired kernel, else 128) and `tiles_per_wave` how many are in flight.  For kernels 2
+ * to 512 rows in the swapped paired kernel, else 128) and `tiles_per_wave` how many are in flight.  For kernels 2
  * and 3 `splits` counts pairs of thread blocks. */
 int pvf_score_plan_for_shape(int32_t vocab, int32_t hidden, int32_t n_sm, int32_t M, int32_t *ctas, int32_t *splits,
                              int32_t *waves, int32_t *kernel, int32_t *row_tiles, int32_t *tiles_per_wave);
 
 /* Name of the projection kernel pvf_score launches for M rows (for profiler filters and reports):
  * "pvf_score_stream_kernel" up to 32 rows (vocabulary on the accumulator lanes, rows on its columns),
- * "pvf_score_swap_pair_kernel" for 33 .. 64 and 129 .. 192 rows (the same layout, two thread blocks per
+ * "pvf_score_swap_pair_kernel" for 33 .. 64, 129 .. 192 and 257 .. 448 rows (the same layout, two thread blocks per
  * vocabulary tile), "pvf_score_gemm_kernel" or "pvf_score_gemm_pair_kernel" otherwise (rows on the lanes).
  * NULL on an invalid argument. */
 const char *pvf_score_kernel_name(pvf_ctx *ctx, int32_t M);
@@ -351,7 +351,7 @@ int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hid
 
 /*
  * pvf_score_static -- pvf_score for callers that must not allocate.  (The paper has no counterpart: this
- * is a packaging variant of pvf_score, same arithmetic, same kernels.)
+ * is a packaging variant of pvf_score: same arithmetic, the same kernels.)
  *
  * Some callers of this library cannot call cudaMalloc at the point where they score: code that runs
  * inside a memory-pool or arena discipline where every device byte is accounted for up front, plugins
@@ -361,6 +361,9 @@ int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hid
  * workspace.  Its scratch memory -- the per-vocabulary-range softmax states that the GEMM kernel writes and
  * the merge kernel reads -- is a fixed 512.25 KiB array inside the library image.  Every GPU that loads
  * the library holds that array until the process exits, whether or not this function is ever called.
+ * (The array holds one state per row and SM.  Where pvf_score would pick the kernel that leaves two, and they
+ * do not fit -- more than 221 rows -- this entry point takes the kernel pvf_score uses outside that window:
+ * same arithmetic, results equal within the accumulation order.)
  *
  *   w_head       device, bf16 [vocab][hidden_size] row-major, 16-byte aligned
  *   hidden       device, bf16 [M][hidden_size], 16-byte aligned; hidden_size a multiple of 8

@@ -57,7 +57,8 @@ struct pvf_score_geometry {
     int stages;      // swapped: pipeline stages that fit the shared-memory ring
     int parts;       // partial states per row handed to the merge kernel (splits, or 2 * splits when swapped)
 };
-pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm);
+// allow_swapped = false leaves the swapped paired kernel (which writes twice as many partial states per row) out.
+pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool allow_swapped = true);
 size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm);
 int pvf_score_init(pvf_ctx *ctx);   // tensor maps of W, kernel attributes
 

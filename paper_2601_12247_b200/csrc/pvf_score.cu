@@ -20,7 +20,8 @@
 // with at most 32 rows take a kernel with the operands swapped
 // (pvf_score_stream_kernel): vocabulary on the lanes, rows on the columns, so that no tensor work is
 // spent on padding rows.  33 .. 64 and 129 .. 192 rows, where 128- and 256-row tiles would be mostly
-// padding, take the paired kernel with swapped operands (pvf_score_swap_pair_kernel).
+// padding, and 257 .. 448 rows, where they sweep W through the SMs twice or more, take the paired kernel
+// with swapped operands (pvf_score_swap_pair_kernel).
 //
 // Work split.  Rows form tiles of 128, the vocabulary granules of 16 entries.  `mb` row tiles are
 // in flight at once, each swept by `splits` blocks over disjoint vocabulary ranges (mb * splits
@@ -175,8 +176,13 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
     const bool timed = ev_start && ev_stop;
     if (timed && cudaEventRecord(ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
     cudaError_t e;
-    if (g.swapped)
-        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(kThreads), kSwapSmemBytes, s, tm_h, maps, a);
+    if (g.swapped) {
+        CUtensorMap tm_h1 = tm_h;                                   // rows 256 .. of H: the second column group, if any
+        if (g.n_pad > kSwapGroupCols &&
+            (rc = make_tensor_map(&tm_h1, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)((g.n_pad - kSwapGroupCols) / 2))) != PVF_OK)
+            return rc;
+        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(kSwapThreads), kSwapSmemBytes, s, tm_h, tm_h1, maps, a);
+    }
     else if (g.paired)
         e = pvf_launch_cluster2(pvf_score_gemm_pair_kernel, dim3(g.ctas), dim3(kThreads), kPairSmemBytes, s, tm_h, maps, a);
     else if (g.streaming)
@@ -231,7 +237,7 @@ SplitPlan plan_split(int M, int V, int D, int workers, int tile_rows, int unit, 
 
 }  // namespace
 
-pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm)
+pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool allow_swapped)
 {
     pvf_score_geometry g;
     const int tiles128 = (M + kTileM - 1) / kTileM;
@@ -248,14 +254,14 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm)
         if (pp.waves > 0 && pp.cost <= 1.05 * p.cost) { p = pp; g.paired = 1; }
     }
     g.swapped = 0; g.n_pad = 0; g.stages = 0;
-    if (n_sm >= 2 && ((M > kStreamRows && M <= PVF_SWAP_SMALL_MAX_ROWS) || (M > kTileM && M <= PVF_SWAP_RAGGED_MAX_ROWS))) {
-        // Swapped paired kernel: one row tile padded to a multiple of 32 rows (the MMA's N), every pair of SMs
-        // sweeps one vocabulary range.  Chosen where the other kernels would pad the rows most (see the kernel).
+    if (allow_swapped && n_sm >= 2 && ((M > kStreamRows && M <= PVF_SWAP_SMALL_MAX_ROWS) || (M > kTileM && M <= PVF_SWAP_RAGGED_MAX_ROWS) ||
+                      (M > kSwapGroupCols && M <= PVF_SWAP_WIDE_MAX_ROWS))) {
+        // Swapped paired kernel: all rows, padded to a multiple of 32, are accumulator columns; every pair of SMs
+        // sweeps one vocabulary range.  Chosen where the other kernels pad the rows most or sweep W twice (see the kernel).
         g.swapped = 1; g.paired = 0;
         g.n_pad = ((M + 31) / 32) * 32;
-        g.a_rows = g.n_pad / 2;
-        const int stage_bytes = kSwapWBytes + (g.n_pad / 2) * kRowBytes;
-        g.stages = kSwapRingBytes / stage_bytes < kSwapMaxStages ? kSwapRingBytes / stage_bytes : kSwapMaxStages;
+        g.a_rows = (g.n_pad < kSwapGroupCols ? g.n_pad : kSwapGroupCols) / 2;     // H box of the first column group
+        g.stages = swap_stages(g.n_pad);
         p.m_tiles = 1; p.mb = 1; p.waves = 1;
         p.units = (V + kPairUnit - 1) / kPairUnit;
         p.splits = n_sm / 2 < p.units ? n_sm / 2 : p.units;
@@ -273,10 +279,11 @@ size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm)
     const int max_tiles = (shape->max_rows + kTileM - 1) / kTileM;
     // Within one kernel choice and row-tile count the need grows with the rows, so it peaks at the upper end of
     // every 128-row step and of the swapped paired kernel's two windows.
-    for (int t = 1; t <= max_tiles + 2; ++t) {
+    for (int t = 1; t <= max_tiles + 3; ++t) {
         int rows = t * kTileM;
         if (t == max_tiles + 1) rows = PVF_SWAP_SMALL_MAX_ROWS;
         if (t == max_tiles + 2) rows = PVF_SWAP_RAGGED_MAX_ROWS;
+        if (t == max_tiles + 3) rows = PVF_SWAP_WIDE_MAX_ROWS;
         if (rows > shape->max_rows) rows = shape->max_rows;
         if (rows <= 0) continue;
         const pvf_score_geometry g = pvf_score_geometry_for(rows, shape->vocab, shape->hidden, n_sm);
@@ -413,7 +420,9 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     StaticDeviceState *st = nullptr;
     int rc = static_device_state(&st);
     if (rc != PVF_OK) return rc;
-    const pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden_size, st->n_sm);
+    pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden_size, st->n_sm);
+    if ((size_t)M * g.parts * sizeof(float4) > kStaticPartialsBytes)       // the array is sized for one state per row and SM:
+        g = pvf_score_geometry_for(M, vocab, hidden_size, st->n_sm, false); // above 221 rows the swapped kernel's two do not fit
     if ((size_t)M * g.parts * sizeof(float4) > kStaticPartialsBytes) return PVF_ERR_TOO_LARGE;
 
     CUtensorMap w_levels[kWBoxSizes];

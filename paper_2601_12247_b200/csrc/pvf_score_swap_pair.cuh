@@ -8,18 +8,28 @@
 namespace {
 
 // ---------------------------------------------------------------------------------- swapped paired kernel
-// 33 .. 256 rows in one row tile: the launch sits at the ridge, where HBM, the tensor pipe and the power cap all
-// matter, and 128- or 256-row MMAs over a ragged row count waste tensor work (and with it clock).  Here the
-// operands of the paired kernel change places: the two blocks of a pair hold 2 x 128 vocabulary entries on
-// their accumulator lanes (each loads its own 128-entry W tile, so W still crosses L2 -> SM once) and the
-// scored rows are the N columns, N = the row tile padded to 32 (each block loads half of the H tile):
+// A few dozen to a few hundred rows: the launch sits at the ridge, where HBM, the L2 -> SM feed, the tensor pipe
+// and the power cap all matter, and 128- or 256-row MMAs over a ragged row count waste tensor work (and with it
+// clock).  Here the operands of the paired kernel change places: the two blocks of a pair hold 2 x 128 vocabulary
+// entries on their accumulator lanes (each loads its own 128-entry W tile, so W still crosses L2 -> SM once) and
+// the scored rows are the N columns, padded to a multiple of 32 (each block loads half of the H rows):
 //     D[v][m] = sum_k W[v][k] * H[m][k],   one 256 x N x 16 MMA (cta_group::2) per 16 elements of k.
-// At most 31 padded rows are wasted.  Measured against the other two kernels (each alone for seconds, so that
-// the power cap has settled, and in short bursts) it wins where they pad most: 33 .. 64 rows (4 .. 5 %) and
-// 129 .. 192 rows (4 .. 9 %); with full 128- or 256-row tiles they are 3 .. 9 % faster, so the geometry picks it
-// for those two windows only.
+// Up to 256 rows are one column group and two accumulators alternate.  257 .. 512 rows are two column groups
+// (256 + the rest: two MMAs per k-step on the same W tile) in ONE accumulator that fills tensor memory, so the
+// epilogue of a vocabulary tile and the MMAs of the next no longer overlap -- still better than sweeping W
+// through the SMs once per 128- or 256-row tile, which is what bounds the other kernels there (their L2 -> SM
+// traffic is 2.3 x this kernel's at 288 rows).
+// Measured against the other kernels (each alone for seconds, so that the power cap has settled, and in short
+// bursts) it wins where they pad most or sweep W twice: 33 .. 64 rows (4 .. 5 %), 129 .. 192 rows (4 .. 9 %) and
+// 257 .. 448 rows (17 % at 257, 7 % at 448); with full 128-, 256- or 512-row tiles they are as fast or 3 .. 9 %
+// faster, so the geometry picks it for those three windows only.
 //
-// Epilogue: a warp owns 32 vocabulary lanes and reads 32 rows (columns) at a time.  It turns that 32 x 32 block
+// The MMA-issuing thread is the most latency-sensitive part: a data-dependent branch between the MMAs of a
+// k-step (one loop serving one or two column groups) cost 17 .. 33 % of the whole launch; the two cases are
+// separate loops.
+//
+// Epilogue: eight warps, two per quadrant of 32 vocabulary lanes, each taking every other group of 32 rows
+// (columns).  A warp turns its 32 x 32 block
 // around through a padded shared-memory tile of its own, after which lane i holds row i's 32 logits and folds
 // them into the running state of row chunk*32 + i exactly as the GEMM kernels' epilogue does (no warp-wide
 // reductions: those serialise on their latency with one epilogue warp per scheduler).  At the end of the block's
@@ -28,33 +38,49 @@ namespace {
 //
 // The ring has as many stages as fit: a stage is the block's 16 KiB W tile plus its half of the H tile.
 constexpr int kSwapWBytes = kTileM * kRowBytes;                      // 16 KiB
-constexpr int kSwapMaxRowsPerTile = 256;                             // MMA N limit
-constexpr int kSwapTmemCols = 512;                                   // 2 accumulators x 256 columns
-constexpr int kSwapTurnPitch = 36;                                   // words per lane of a warp's 32 x 32 fp32 block: 16-byte
-                                                                     // aligned rows, conflict-free 128-bit stores and column reads
-constexpr int kSwapWarpScratchBytes = 32 * kSwapTurnPitch * 4;       // that block; later the warp's 256 row states (4 KiB) for the fold
-constexpr int kSwapScratchBytes = 4 * kSwapWarpScratchBytes;
-static_assert(kSwapWarpScratchBytes >= kSwapMaxRowsPerTile * 16 && kSwapWarpScratchBytes % 16 == 0, "fold scratch");
-constexpr int kSwapRingBytes = 204 * 1024;
+constexpr int kSwapGroupCols = 256;                                  // MMA N limit: columns (rows of H) per MMA
+constexpr int kSwapMaxRows = 512;                                    // two column groups fill tensor memory
+constexpr int kSwapTmemCols = 512;                                   // two accumulators of up to 256 columns, or one of up to 512
+constexpr int kSwapEpilogueWarps = 8;                                // two per tensor-memory lane quadrant, taking alternate row chunks
+constexpr int kSwapEpilogueThreads = kSwapEpilogueWarps * 32;
+constexpr int kSwapThreads = 64 + kSwapEpilogueThreads;              // producer warp, MMA warp, epilogue warps
+constexpr int kSwapTurnPitch = 33;                                   // words per lane of a warp's 32 x 32 fp32 block (conflict-free both ways)
+constexpr int kSwapWarpScratchBytes = 32 * kSwapTurnPitch * 4;       // that block, one per epilogue warp
+constexpr int kSwapQuadScratchBytes = 2 * kSwapWarpScratchBytes;     // the two warps of a quadrant; at the end the quadrant's row states
+constexpr int kSwapScratchBytes = 4 * kSwapQuadScratchBytes;
 constexpr int kSwapMaxStages = 12;
-constexpr int kSwapSmemBytes = kSwapRingBytes + 1024 + 512 + kSwapScratchBytes;
-static_assert(kSwapSmemBytes <= 227 * 1024, "swapped ring");
+constexpr int kSwapSmemBytes = 227 * 1024;                           // everything: alignment slack, ring, control block, scratch
+static_assert(kSwapQuadScratchBytes >= kSwapMaxRows * 16 && kSwapQuadScratchBytes % 16 == 0, "fold scratch");
 static_assert(kSwapMaxStages <= kMaxStages, "barrier arrays");
-static_assert(PVF_SWAP_SMALL_MAX_ROWS <= kSwapMaxRowsPerTile && PVF_SWAP_RAGGED_MAX_ROWS <= kSwapMaxRowsPerTile, "one row tile");
+static_assert(PVF_SWAP_SMALL_MAX_ROWS <= kSwapGroupCols && PVF_SWAP_RAGGED_MAX_ROWS <= kSwapGroupCols &&
+              PVF_SWAP_WIDE_MAX_ROWS <= kSwapMaxRows, "row limits");
 
-__global__ void __launch_bounds__(kThreads, 1)
-pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ WMaps tm_w, const ScoreArgs args)
+__host__ __device__ constexpr int swap_stage_bytes(int n_pad) { return kSwapWBytes + (n_pad / 2) * kRowBytes; }
+// Pipeline stages that fit beside the control block and the epilogue's scratch.
+inline int swap_stages(int n_pad)
+{
+    const int ring = kSwapSmemBytes - 1024 - 512 - kSwapScratchBytes;
+    const int n = ring / swap_stage_bytes(n_pad);
+    return n < kSwapMaxStages ? n : kSwapMaxStages;
+}
+
+__global__ void __launch_bounds__(kSwapThreads, 1)
+pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ CUtensorMap tm_h1,
+                           const __grid_constant__ WMaps tm_w, const ScoreArgs args)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t tiles_addr = (raw_addr + 1023u) & ~1023u;
     uint8_t *tiles_ptr = smem_raw + (tiles_addr - raw_addr);
-    const int n_pad = args.n_pad;                                        // rows per row tile = MMA N (multiple of 32)
+    const int n_pad = args.n_pad;                                        // padded rows = accumulator columns (multiple of 32)
+    const int n0 = min(n_pad, kSwapGroupCols), n1 = n_pad - n0;          // columns of the first and the second MMA of a k-step
+    const int n_bufs = n1 > 0 ? 1 : 2;                                   // accumulators: two alternate while they fit
     const int n_stages = args.stages;
-    const uint32_t h_bytes = (uint32_t)(n_pad / 2) * kRowBytes;          // this block's half of the H tile
-    const uint32_t stage_bytes = (uint32_t)kSwapWBytes + h_bytes;
+    const uint32_t h0_bytes = (uint32_t)(n0 / 2) * kRowBytes;            // this block's half of each column group's H rows
+    const uint32_t h1_bytes = (uint32_t)(n1 / 2) * kRowBytes;
+    const uint32_t stage_bytes = (uint32_t)kSwapWBytes + h0_bytes + h1_bytes;
     SharedControl *ctl = reinterpret_cast<SharedControl *>(tiles_ptr + (size_t)n_stages * stage_bytes);
-    uint8_t *scratch = reinterpret_cast<uint8_t *>(ctl) + 512;          // one kSwapWarpScratchBytes region per epilogue warp
+    uint8_t *scratch = reinterpret_cast<uint8_t *>(ctl) + 512;          // kSwapScratchBytes
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -66,9 +92,10 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     const int n_tiles = split.n_tiles;
     const int k_steps = args.num_kb;
 
-    if (threadIdx.x == 0) init_pipeline_barriers(ctl, n_stages, 1, 2 * kEpilogueThreads);
+    if (threadIdx.x == 0) init_pipeline_barriers(ctl, n_stages, 1, 2 * kSwapEpilogueThreads);
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h1) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_w.size[kPairUnitsPerTile - 1]) : "memory");
     }
     if (warp == 1) {
@@ -89,11 +116,12 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             int stage = 0;
             uint32_t phase = 0;
             bool alive = true;
-            const int row0 = (int)rank * (n_pad / 2);                               // this block's half of the rows
+            const int row0 = (int)rank * (n0 / 2);                                  // this block's half of each group's rows
+            const int row1 = n0 + (int)rank * (n1 / 2);
             for (int tile = 0; tile < n_tiles && alive; ++tile) {
                 int tu0, tun;
                 split.tile(tile, &tu0, &tun);
-                const uint32_t bytes = 2u * ((uint32_t)tun * kUnitBytes + h_bytes);                     // both blocks
+                const uint32_t bytes = 2u * ((uint32_t)tun * kUnitBytes + h0_bytes + h1_bytes);         // both blocks
                 const int w_row = tu0 * kPairUnit + (int)rank * tun * kUnit;                            // this block's entries
                 for (int step = 0; step < k_steps; ++step) {
                     if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
@@ -102,6 +130,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
                     if (rank == 0) mbar_arrive_expect_tx(full, bytes);
                     tma_load_2d_pair(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
                     tma_load_2d_pair(w_dst + kSwapWBytes, &tm_h, full, step * kBlockK, row0);
+                    if (n1 > 0) tma_load_2d_pair(w_dst + kSwapWBytes + h0_bytes, &tm_h1, full, step * kBlockK, row1);
                     if (++stage == n_stages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -116,24 +145,36 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             int stage = 0;
             uint32_t phase = 0;
             bool alive = true;
-            const uint32_t idesc = instr_desc_bf16_m256(n_pad);
+            const uint32_t idesc0 = instr_desc_bf16_m256(n0);
+            const uint32_t idesc1 = instr_desc_bf16_m256(n1 > 0 ? n1 : n0);
             for (int tile = 0; tile < n_tiles && alive; ++tile) {
-                const uint32_t buf = (uint32_t)tile & 1u;
-                const uint32_t acc_phase = ((uint32_t)tile >> 1) & 1u;
+                const uint32_t buf = n_bufs == 2 ? ((uint32_t)tile & 1u) : 0u;
+                const uint32_t acc_phase = (n_bufs == 2 ? ((uint32_t)tile >> 1) : (uint32_t)tile) & 1u;
                 if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), acc_phase ^ 1u, ctl, args.status)) { alive = false; break; }
                 tc_fence_after_sync();
-                const uint32_t tmem_d = tmem_base + buf * kSwapMaxRowsPerTile;
+                const uint32_t tmem_d = tmem_base + buf * kSwapGroupCols;
                 for (int step = 0; step < k_steps; ++step) {
                     if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, ctl, args.status)) { alive = false; break; }
                     tc_fence_after_sync();
                     // A ragged vocabulary tile leaves stale bytes on the W tile's last rows: lanes the epilogue skips.
                     const uint32_t w_addr = tiles_addr + (uint32_t)stage * stage_bytes;
                     const uint64_t w_desc = smem_desc_k_major_sw128(w_addr);
-                    const uint64_t h_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes);
+                    const uint64_t h0_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes);
+                    const uint64_t h1_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes + h0_bytes);
+                    if (n1 == 0) {
 #pragma unroll
-                    for (int k = 0; k < kBlockK / 16; ++k)
-                        tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h_desc + (uint64_t)(k * 2), idesc,
-                                         (step | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < kBlockK / 16; ++k)
+                            tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h0_desc + (uint64_t)(k * 2), idesc0,
+                                             (step | k) != 0 ? 1u : 0u);
+                    } else {                                     // columns 256 .. : the second group of rows, same W tile
+#pragma unroll
+                        for (int k = 0; k < kBlockK / 16; ++k) {
+                            tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h0_desc + (uint64_t)(k * 2), idesc0,
+                                             (step | k) != 0 ? 1u : 0u);
+                            tc_mma_bf16_pair(tmem_base + kSwapGroupCols, w_desc + (uint64_t)(k * 2), h1_desc + (uint64_t)(k * 2),
+                                             idesc1, (step | k) != 0 ? 1u : 0u);
+                        }
+                    }
                     tc_commit_pair(smem_u32(&ctl->empty[stage]));
                     if (++stage == n_stages) { stage = 0; phase ^= 1u; }
                 }
@@ -148,20 +189,22 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     } else {
         // ------------------------------------------------------------------ softmax epilogue (both blocks)
         const int quad = warp & 3;                                       // tensor-memory lanes quad*32 .. quad*32+31
+        const int half = (warp - 2) >> 2;                                // which of the quadrant's two warps: takes row chunks
+                                                                         // half, half + 2, half + 4, ...
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int n_chunks = n_pad >> 5;                                 // 32-row column groups
-        const int e_thread = quad * 32 + lane;
-        float *turn = reinterpret_cast<float *>(scratch + quad * kSwapWarpScratchBytes);          // [32 lanes][kSwapTurnPitch]
-        float4 *fold_mine = reinterpret_cast<float4 *>(scratch + quad * kSwapWarpScratchBytes);   // [256 rows], after the sweep
+        const int e_thread = (int)threadIdx.x - 64;                      // 0 .. 255
+        float *turn = reinterpret_cast<float *>(scratch + quad * kSwapQuadScratchBytes + half * kSwapWarpScratchBytes);
+        float4 *fold_quad = reinterpret_cast<float4 *>(scratch + quad * kSwapQuadScratchBytes);   // [n_pad rows], after the sweep
         bool alive = true;
-        RowState st[kSwapMaxRowsPerTile / 32];                           // lane i: state of row chunk*32 + i
+        RowState st[kSwapMaxRows / 64];                                  // st[i], lane l: state of row (2 i + half) * 32 + l
 #pragma unroll
-        for (int c = 0; c < kSwapMaxRowsPerTile / 32; ++c) { st[c].m = -INFINITY; st[c].s = 0.f; st[c].t = 0.f; st[c].arg = kNoArg; }
+        for (int i = 0; i < kSwapMaxRows / 64; ++i) { st[i].m = -INFINITY; st[i].s = 0.f; st[i].t = 0.f; st[i].arg = kNoArg; }
         for (int tile = 0; tile < n_tiles && alive; ++tile) {
             int tu0, tun;
             split.tile(tile, &tu0, &tun);
-            const uint32_t buf = (uint32_t)tile & 1u;
-            const uint32_t acc_phase = ((uint32_t)tile >> 1) & 1u;
+            const uint32_t buf = n_bufs == 2 ? ((uint32_t)tile & 1u) : 0u;
+            const uint32_t acc_phase = (n_bufs == 2 ? ((uint32_t)tile >> 1) : (uint32_t)tile) & 1u;
             if (!mbar_wait(smem_u32(&ctl->acc_full[buf]), acc_phase, ctl, args.status)) { alive = false; break; }
             tc_fence_after_sync();
             const int block_v0 = tu0 * kPairUnit + (int)rank * tun * kUnit;         // vocabulary id on this block's lane 0
@@ -170,29 +213,29 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             const int n_real = min(32, block_end - warp_v0);                        // vocabulary entries on this warp's lanes
             if (n_real > 0) {                                                        // warp-uniform
 #pragma unroll
-                for (int c = 0; c < kSwapMaxRowsPerTile / 32; ++c) {
-                    if (c < n_chunks) {                                              // block-uniform
+                for (int i = 0; i < kSwapMaxRows / 64; ++i) {
+                    const int c = 2 * i + half;
+                    if (c < n_chunks) {                                              // warp-uniform
                         uint32_t lo[16], hi[16];
-                        const uint32_t col = lane_addr + buf * kSwapMaxRowsPerTile + c * 32;
+                        const uint32_t col = lane_addr + buf * kSwapGroupCols + c * 32;       // column = row: group 1 starts at 256
                         tmem_ld16(col, lo);
                         tmem_ld16(col + 16, hi);
                         tmem_ld_wait();
-                        uint4 *mine = reinterpret_cast<uint4 *>(turn + lane * kSwapTurnPitch);       // lane = vocabulary entry
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            mine[j] = make_uint4(lo[4 * j], lo[4 * j + 1], lo[4 * j + 2], lo[4 * j + 3]);
-                            mine[4 + j] = make_uint4(hi[4 * j], hi[4 * j + 1], hi[4 * j + 2], hi[4 * j + 3]);
+                        for (int j = 0; j < 16; ++j) {                               // lane = vocabulary entry, j = row
+                            turn[lane * kSwapTurnPitch + j] = __uint_as_float(lo[j]);
+                            turn[lane * kSwapTurnPitch + 16 + j] = __uint_as_float(hi[j]);
                         }
                         __syncwarp();
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {                       // lane = row, 16 vocabulary entries at a time
-                            const int n = n_real - half * 16;
+                        for (int part = 0; part < 2; ++part) {                       // lane = row, 16 vocabulary entries at a time
+                            const int n = n_real - part * 16;
                             if (n > 0) {
                                 uint32_t x[16];
 #pragma unroll
-                                for (int l = 0; l < 16; ++l) x[l] = __float_as_uint(turn[(half * 16 + l) * kSwapTurnPitch + lane]);
-                                if (n >= 16) fold16<true>(st[c], x, warp_v0 + half * 16, 16);
-                                else fold16<false>(st[c], x, warp_v0 + half * 16, n);
+                                for (int l = 0; l < 16; ++l) x[l] = __float_as_uint(turn[(part * 16 + l) * kSwapTurnPitch + lane]);
+                                if (n >= 16) fold16<true>(st[i], x, warp_v0 + part * 16, 16);
+                                else fold16<false>(st[i], x, warp_v0 + part * 16, n);
                             }
                         }
                         __syncwarp();
@@ -202,21 +245,25 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             tc_fence_before_sync();
             mbar_arrive_even_block(smem_u32(&ctl->acc_empty[buf]));
         }
-        // Fold the block's four warps and write the block's partial state of every row.  Every epilogue thread
-        // reaches the barrier, aborting or not.
+        // Fold the block's four quadrants and write the block's partial state of every row.  The row states
+        // reuse the turn tiles, so every warp must have left its last tile first.  Every epilogue thread reaches
+        // the barriers, aborting or not.
+        asm volatile("bar.sync 1, %0;" ::"n"(kSwapEpilogueThreads) : "memory");
         if (alive) {
 #pragma unroll
-            for (int c = 0; c < kSwapMaxRowsPerTile / 32; ++c)
+            for (int i = 0; i < kSwapMaxRows / 64; ++i) {
+                const int c = 2 * i + half;
                 if (c < n_chunks)
-                    fold_mine[c * 32 + lane] = make_float4(st[c].m, st[c].s, st[c].t, __int_as_float(st[c].arg));
+                    fold_quad[c * 32 + lane] = make_float4(st[i].m, st[i].s, st[i].t, __int_as_float(st[i].arg));
+            }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kEpilogueThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"n"(kSwapEpilogueThreads) : "memory");
         if (alive && !ctl->abort_flag) {
-            for (int row = e_thread; row < args.M; row += kEpilogueThreads) {
+            for (int row = e_thread; row < args.M; row += kSwapEpilogueThreads) {
                 float4 acc = reinterpret_cast<const float4 *>(scratch)[row];
 #pragma unroll
                 for (int o = 1; o < 4; ++o)
-                    state_merge(acc, reinterpret_cast<const float4 *>(scratch + o * kSwapWarpScratchBytes)[row]);
+                    state_merge(acc, reinterpret_cast<const float4 *>(scratch + o * kSwapQuadScratchBytes)[row]);
                 args.partials[(size_t)row * args.parts + 2 * q + (int)rank] = acc;
             }
         }

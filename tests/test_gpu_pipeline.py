@@ -222,17 +222,19 @@ def test_second_model_shape_sampled():
     plan = synth.make_plan_ids(1005, V, 2048)
     ctx = make_ctx(w_bits, plan, 512, 8, 8)
     st = synth.config1("b", stress=True, w_bits=w_bits, vocab=V, hidden=D)
+    h_bits = np.concatenate([st.h_bits, st.h_bits[:64][::-1]])            # 320 rows: the last 64 repeat earlier ones
     for rows, kernel, sample in ((32, "pvf_score_stream_kernel", np.array([0, 1, 15, 16, 30, 31])),
                                  (48, "pvf_score_swap_pair_kernel", np.array([0, 23, 24, 32, 47])),
                                  (100, "pvf_score_gemm_kernel", np.array([0, 31, 32, 64, 99])),
                                  (170, "pvf_score_swap_pair_kernel", np.array([0, 95, 96, 128, 169])),
-                                 (256, "pvf_score_gemm_pair_kernel", np.array([0, 127, 128, 129, 255]))):
+                                 (256, "pvf_score_gemm_pair_kernel", np.array([0, 127, 128, 129, 255])),
+                                 (300, "pvf_score_swap_pair_kernel", np.array([0, 127, 128, 255, 256, 277, 278, 299]))):
         assert ctx.score_kernel_name(rows) == kernel
-        got = to_np(ctx.score(upload_bits(st.h_bits[:rows])))
+        got = to_np(ctx.score(upload_bits(h_bits[:rows])))
         torch.cuda.synchronize()
         assert ctx.last_status() == 0
         check_score_properties(got, V, plan)
-        check_score(got, oscore.score(w_bits, st.h_bits[sample], plan), V, plan, rows=sample)
+        check_score(got, oscore.score(w_bits, h_bits[sample], plan), V, plan, rows=sample)
     ctx.close()
 
 

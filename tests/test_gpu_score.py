@@ -40,12 +40,13 @@ def test_config0_tiny(stress):
                                    (4096, 256, 16), (4096, 256, 17), (4096, 256, 31), (4096, 256, 32),
                                    (5000, 200, 20), (70000, 512, 30), (100, 64, 5), (300, 72, 9), (40000, 136, 32),
                                    (4096, 256, 40), (5000, 200, 64), (300, 72, 50), (70000, 512, 160), (40000, 136, 191),
-                                   (5000, 200, 192), (100, 64, 130), (4100, 256, 65), (4100, 256, 193)])
+                                   (5000, 200, 192), (100, 64, 130), (4100, 256, 65), (4100, 256, 193),
+                                   (4096, 256, 257), (5000, 200, 290), (70000, 512, 448), (300, 72, 449), (40000, 136, 400)])
 def test_ragged_shapes(V, D, M):
     # several row tiles, vocabulary not a multiple of 16 or 32, hidden size not a multiple of 64; up to 32 rows take
-    # the swapped-operand streaming kernel, 33 .. 64 and 129 .. 192 rows the swapped paired kernel (its row tile
-    # padded to 64, 160 or 192 rows; vocabularies of fewer granules than pairs of SMs), other counts the
-    # 128-row GEMM kernel or the paired kernel
+    # the swapped-operand streaming kernel, 33 .. 64, 129 .. 192 and 257 .. 448 rows the swapped paired kernel (rows
+    # padded to a multiple of 32; above 256 in two column groups; vocabularies of fewer granules than pairs of
+    # SMs), other counts the 128-row GEMM kernel or the paired kernel
     pos = np.arange(M)
     st = synth.build_step("ragged", 4242, V, D, min(64, V), [(pos, np.ones(M, np.uint8))], M, M,
                           dict(tau_high=0.9, budget=4), amp_max=40.0 * (256.0 / D) ** 0.5)
@@ -81,7 +82,7 @@ def test_exact_tie_goes_to_lowest_id_across_ranges():
     ctx.close()
 
 
-@pytest.mark.parametrize("M", [1, 20, 40, 100, 150])
+@pytest.mark.parametrize("M", [1, 20, 40, 100, 150, 300])
 def test_exact_ties_inside_one_range(M):
     # equal logits at ids that one block sees on the same accumulator lane (10 and 138), in its other
     # 128-entry slice (138), in a later tile (300) and in another block's range (60000)
@@ -93,13 +94,13 @@ def test_exact_ties_inside_one_range(M):
     h = np.zeros((M, D), np.float32)
     h[:] = synth.bf16_bits_to_f32(w[10]).astype(np.float32) * 400.0
     h[M - 1] = synth.bf16_bits_to_f32(w[19999]).astype(np.float32) * 400.0
-    ctx = make_ctx(w, [10], 256)
+    ctx = make_ctx(w, [10], 512)
     got = to_np(ctx.score(upload_bits(synth.f32_to_bf16_bits(h))))
     assert (got["tok"][:M - 1] == 10).all() and got["tok"][M - 1] == 19999
     ctx.close()
 
 
-@pytest.mark.parametrize("max_rows", [33, 64, 100, 129, 192, 200, 300])
+@pytest.mark.parametrize("max_rows", [33, 64, 100, 129, 192, 200, 300, 448, 460, 600])
 def test_workspace_covers_every_row_count_up_to_max_rows(max_rows):
     # the kernels leave a different number of partial states per row (148 in the swapped paired kernel's windows,
     # 74 just above them): a context sized for max_rows must serve every smaller call
@@ -107,7 +108,7 @@ def test_workspace_covers_every_row_count_up_to_max_rows(max_rows):
     w = synth.make_w(5, V, D)
     ctx = make_ctx(w, [1], max_rows)
     h = upload_bits(synth.make_w(6, max_rows, D))
-    for M in sorted({1, 32, 33, 64, 65, 128, 129, 192, 193, 256, max_rows}):
+    for M in sorted({1, 32, 33, 64, 65, 128, 129, 192, 193, 256, 257, 448, 449, 512, max_rows}):
         if M <= max_rows:
             out = ctx.score(h[:M])
             assert out["tok"].shape[0] == M
@@ -161,15 +162,15 @@ def test_non_finite_hidden_rows_stay_in_bounds_and_do_not_disturb_other_rows(M):
     ctx.close()
 
 
-@pytest.mark.parametrize("copies", [1, 2, 32, 256])
+@pytest.mark.parametrize("copies", [1, 2, 5, 32, 256])
 def test_small_tail_terms_are_not_lost_beside_a_dominant_logit(copies):
     # One logit 11 .. 20 above a narrow bulk (hidden size 1024: the other logits spread by 0.5 only): every other
     # term e^{x - max} is near or below the fp32 rounding unit of 1.0, yet there are 70000 of them and together
     # they hold up to a per cent of the probability mass.  A running sum that contains the dominant term's 1.0
     # rounds them away -- the more, the longer the vocabulary range one block sweeps, i.e. the more rows the call
     # has: 64 distinct rows are scored once (swapped paired kernel, 74 ranges), twice over (128 rows: 128-row
-    # kernel, 148 ranges), 32 times over (2048 rows, paired kernel) and 256 times over (16384 rows, few ranges per
-    # row tile).
+    # kernel, 148 ranges), 5 times over (320 rows: swapped paired kernel in two column groups), 32 times over (2048
+    # rows, paired kernel) and 256 times over (16384 rows, few ranges per row tile).
     V, D, M = 70000, 1024, 64
     w = synth.make_w(21, V, D)
     targets = (np.arange(M) * 331 + 7) % V

@@ -10,13 +10,13 @@ SHAPES = [(126464, 4096), (152064, 3584), (4096, 256), (100, 64), (16, 8), (7000
 @pytest.mark.parametrize("V,D", SHAPES)
 @pytest.mark.parametrize("n_sm", [148, 132, 2, 1])
 def test_plan_covers_the_work(V, D, n_sm):
-    rows = list(range(1, 70)) + [96, 127, 128, 129, 160, 191, 192, 193, 224, 255, 256, 257, 300, 511, 512, 513, 1000, 1024, 4096, 8192, 8193,
+    rows = list(range(1, 70)) + [96, 127, 128, 129, 160, 191, 192, 193, 224, 288, 448, 449, 255, 256, 257, 300, 511, 512, 513, 1000, 1024, 4096, 8192, 8193,
                                  13704, 16384, 32768, 103042]
     for M in rows:
         p = binding.score_plan_for_shape(V, D, n_sm, M)
         paired = p["kernel"] in (2, 3)                                            # blocks work in pairs
         granule = 32 if paired else 16
-        if p["kernel"] == 3:                                                      # swapped: one row tile of up to 256 rows
+        if p["kernel"] == 3:                                                      # swapped: one row tile of up to 512 rows
             assert p["row_tiles"] == 1 and p["waves"] == 1 and p["tiles_per_wave"] == 1
         else:
             tile_rows = 256 if p["kernel"] == 2 else 128
@@ -26,7 +26,7 @@ def test_plan_covers_the_work(V, D, n_sm):
         assert 1 <= p["splits"] <= -(-V // granule)                               # no range without a granule
         per_tile = 2 if paired else 1
         assert p["ctas"] == p["tiles_per_wave"] * p["splits"] * per_tile and 1 <= p["ctas"] <= max(n_sm, per_tile)
-        swap_window = 32 < M <= 64 or 128 < M <= 192
+        swap_window = 32 < M <= 64 or 128 < M <= 192 or 256 < M <= 448
         if M <= 32:
             assert p["kernel"] == 0 and p["row_tiles"] == 1 and p["waves"] == 1
         elif n_sm < 2 or M > 8192:
@@ -36,7 +36,7 @@ def test_plan_covers_the_work(V, D, n_sm):
         elif M <= 128:
             assert p["kernel"] == 1
         if p["kernel"] == 2:
-            assert p["ctas"] % 2 == 0 and 192 < M <= 8192
+            assert p["ctas"] % 2 == 0 and 192 < M <= 8192 and not swap_window
         if p["kernel"] == 3:
             assert p["ctas"] % 2 == 0 and swap_window
 
@@ -47,6 +47,7 @@ def test_llada_shape_choices_on_148_sms():
     assert plan(256)["kernel"] == 2 and plan(256)["splits"] == 74 and plan(256)["waves"] == 1
     assert plan(48) == dict(ctas=148, splits=74, waves=1, kernel=3, row_tiles=1, tiles_per_wave=1)
     assert plan(160)["kernel"] == 3 and plan(96)["kernel"] == 1 and plan(200)["kernel"] == 2
+    assert plan(300)["kernel"] == 3 and plan(448)["kernel"] == 3 and plan(449)["kernel"] in (1, 2)
     assert plan(1024)["kernel"] == 2 and plan(1024)["ctas"] == 144
     p = plan(32768)
     assert p["kernel"] == 1 and p["ctas"] == 148 and p["waves"] * p["tiles_per_wave"] >= 256
