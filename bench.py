@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the fused PVF step on one node.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1a|cfg1b|cfg2|cfg3|cfg3s|dream1a|dream1b]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg1a|cfg1b|cfg2|cfg2w|cfg3|cfg3s|dream1a|dream1b]
 
 A step is one pass of the whole hot path over one synthetic batch, through the C interface:
     pvf_score(H) -> pvf_commit -> pvf_select_drafts -> pvf_score(Hv, verification pass) -> pvf_verify
@@ -44,6 +44,7 @@ NCU_TRAFFIC_PER_WAVE = {
     "pvf_score_gemm_pair_kernel": 1.0490e9,
     "pvf_score_swap_pair_kernel": 1.0495e9,
 }
+NCU_TRAFFIC_SWAP_WIDE = 1.0573e9          # the swapped paired kernel above 256 rows (two column groups)
 
 
 def load_peaks():
@@ -68,6 +69,8 @@ def make_workload(name: str, synth, seed_w: int = 1001):
         st = synth.config1("b", w_bits=w_bits)
     elif name == "cfg2":
         st = synth.config2(w_bits=w_bits)
+    elif name == "cfg2w":                 # config 2's recipe at batch 24: both passes score 257 .. 448 rows
+        st = synth.config2(w_bits=w_bits, n_seq=24)
     elif name == "cfg3":
         st = synth.config3(w_bits=w_bits)
     elif name == "cfg3s":                 # 8 of config 3's 64 sequences: the size profiler captures use
@@ -340,7 +343,10 @@ def run_ours(args):
         roof = dict(bound="tensor", achieved=alg_flops / t_gemm / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
     kernels = sorted({ctx.score_kernel_name(r) for _, _, r in ev_pairs})
-    per_launch = [NCU_TRAFFIC_PER_WAVE.get(ctx.score_kernel_name(r)) for _, _, r in ev_pairs]
+    def launch_traffic(rows):
+        name = ctx.score_kernel_name(rows)
+        return NCU_TRAFFIC_SWAP_WIDE if (name == "pvf_score_swap_pair_kernel" and rows > 256) else NCU_TRAFFIC_PER_WAVE.get(name)
+    per_launch = [launch_traffic(r) for _, _, r in ev_pairs]
     if per_launch and all(t is not None for t in per_launch):       # average launch of the timed mix
         traffic = sum(t * ctx.score_plan(r)["waves"] for t, (_, _, r) in zip(per_launch, ev_pairs)) / n_gemm
     else:
@@ -440,7 +446,7 @@ def main():
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg3", "cfg3s", "dream1a", "dream1b"])
+    ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg2w", "cfg3", "cfg3s", "dream1a", "dream1b"])
     ap.add_argument("--cpu-rows", type=int, default=256, help="rows per pass the CPU baseline scores")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay of the step")
