@@ -169,6 +169,17 @@ def test_config2_full_step_on_the_oracles_own_scores(llada):
     ctx.close()
 
 
+def test_config2_at_batch_24_sampled(llada):
+    # config 2's recipe with 24 sequences: 354 rows, which the swapped paired kernel takes in two column groups
+    # (rows 0..255 and 256..383 of one accumulator); sampled on both sides of the group boundary, at the edges of
+    # the 32-row chunks the epilogue warps alternate on, and on the last real row
+    w_bits, plan, ctx = llada
+    st = synth.config2(w_bits=w_bits, n_seq=24)
+    assert 256 < st.n_rows <= 448 and ctx.score_kernel_name(st.n_rows) == "pvf_score_swap_pair_kernel"
+    M = st.n_rows
+    sampled_parity(ctx, st, w_bits, plan, np.array([0, 31, 32, 127, 128, 255, 256, 257, 287, 288, 319, 320, M - 1]))
+
+
 def test_config2_sampled_rows_and_decisions_on_gpu_scores(llada):
     w_bits, plan, ctx = llada
     st = synth.config2(w_bits=w_bits)
