@@ -181,7 +181,7 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
         if (g.n_pad > kSwapGroupCols &&
             (rc = make_tensor_map(&tm_h1, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)((g.n_pad - kSwapGroupCols) / 2))) != PVF_OK)
             return rc;
-        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(kSwapThreads), kSwapSmemBytes, s, tm_h, tm_h1, maps, a);
+        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(64 + 128 * swap_warps_per_quad(g.n_pad)), kSwapSmemBytes, s, tm_h, tm_h1, maps, a);
     }
     else if (g.paired)
         e = pvf_launch_cluster2(pvf_score_gemm_pair_kernel, dim3(g.ctas), dim3(kThreads), kPairSmemBytes, s, tm_h, maps, a);

@@ -41,16 +41,19 @@ constexpr int kSwapWBytes = kTileM * kRowBytes;                      // 16 KiB
 constexpr int kSwapGroupCols = 256;                                  // MMA N limit: columns (rows of H) per MMA
 constexpr int kSwapMaxRows = 512;                                    // two column groups fill tensor memory
 constexpr int kSwapTmemCols = 512;                                   // two accumulators of up to 256 columns, or one of up to 512
-constexpr int kSwapEpilogueWarps = 8;                                // two per tensor-memory lane quadrant, taking alternate row chunks
+constexpr int kSwapEpilogueWarps = 8;                                // launched; one per tensor-memory lane quadrant works on up to 256
+                                                                     // rows, two (taking alternate row chunks) above
 constexpr int kSwapEpilogueThreads = kSwapEpilogueWarps * 32;
 constexpr int kSwapThreads = 64 + kSwapEpilogueThreads;              // producer warp, MMA warp, epilogue warps
 constexpr int kSwapTurnPitch = 33;                                   // words per lane of a warp's 32 x 32 fp32 block (conflict-free both ways)
 constexpr int kSwapWarpScratchBytes = 32 * kSwapTurnPitch * 4;       // that block, one per epilogue warp
-constexpr int kSwapQuadScratchBytes = 2 * kSwapWarpScratchBytes;     // the two warps of a quadrant; at the end the quadrant's row states
-constexpr int kSwapScratchBytes = 4 * kSwapQuadScratchBytes;
+// Scratch of one quadrant = its warps' blocks; at the end it holds the quadrant's row states (16 bytes per row).
+__host__ __device__ constexpr int swap_warps_per_quad(int n_pad) { return n_pad > kSwapGroupCols ? 2 : 1; }
+__host__ __device__ constexpr int swap_quad_scratch_bytes(int n_pad) { return swap_warps_per_quad(n_pad) * kSwapWarpScratchBytes; }
 constexpr int kSwapMaxStages = 12;
 constexpr int kSwapSmemBytes = 227 * 1024;                           // everything: alignment slack, ring, control block, scratch
-static_assert(kSwapQuadScratchBytes >= kSwapMaxRows * 16 && kSwapQuadScratchBytes % 16 == 0, "fold scratch");
+static_assert(swap_quad_scratch_bytes(kSwapMaxRows) >= kSwapMaxRows * 16 && swap_quad_scratch_bytes(kSwapGroupCols) >= kSwapGroupCols * 16 &&
+              kSwapWarpScratchBytes % 16 == 0, "fold scratch");
 static_assert(kSwapMaxStages <= kMaxStages, "barrier arrays");
 static_assert(PVF_SWAP_SMALL_MAX_ROWS <= kSwapGroupCols && PVF_SWAP_RAGGED_MAX_ROWS <= kSwapGroupCols &&
               PVF_SWAP_WIDE_MAX_ROWS <= kSwapMaxRows, "row limits");
@@ -59,9 +62,98 @@ __host__ __device__ constexpr int swap_stage_bytes(int n_pad) { return kSwapWByt
 // Pipeline stages that fit beside the control block and the epilogue's scratch.
 inline int swap_stages(int n_pad)
 {
-    const int ring = kSwapSmemBytes - 1024 - 512 - kSwapScratchBytes;
+    const int ring = kSwapSmemBytes - 1024 - 512 - 4 * swap_quad_scratch_bytes(n_pad);
     const int n = ring / swap_stage_bytes(n_pad);
     return n < kSwapMaxStages ? n : kSwapMaxStages;
+}
+
+// The producer's and the MMA thread's loops, once for one column group (kWide = false) and once for two: these
+// two threads set the pace of the kernel, and a run-time choice inside their loops costs more than it looks.
+struct SwapLoopArgs {
+    uint32_t tiles_addr, stage_bytes, h0_bytes, h1_bytes, tmem_base;
+    int n0, n1, n_stages, n_tiles, k_steps, n_bufs;
+    uint32_t rank;
+};
+
+template <bool kWide>
+__device__ __forceinline__ void swap_produce(const SwapLoopArgs &a, const TileSplit &split, SharedControl *ctl,
+                                             const CUtensorMap *tm_h, const CUtensorMap *tm_h1, const WMaps &tm_w,
+                                             int32_t *status)
+{
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;
+    const int row0 = (int)a.rank * (a.n0 / 2);                                      // this block's half of each group's rows
+    const int row1 = a.n0 + (int)a.rank * (a.n1 / 2);
+    for (int tile = 0; tile < a.n_tiles && alive; ++tile) {
+        int tu0, tun;
+        split.tile(tile, &tu0, &tun);
+        const uint32_t bytes = 2u * ((uint32_t)tun * kUnitBytes + a.h0_bytes + (kWide ? a.h1_bytes : 0u));   // both blocks
+        const int w_row = tu0 * kPairUnit + (int)a.rank * tun * kUnit;                                        // this block's entries
+        for (int step = 0; step < a.k_steps; ++step) {
+            if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, status)) { alive = false; break; }
+            const uint32_t full = smem_u32(&ctl->full[stage]);
+            const uint32_t w_dst = a.tiles_addr + (uint32_t)stage * a.stage_bytes;
+            if (a.rank == 0) mbar_arrive_expect_tx(full, bytes);
+            tma_load_2d_pair(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
+            tma_load_2d_pair(w_dst + kSwapWBytes, tm_h, full, step * kBlockK, row0);
+            if (kWide) tma_load_2d_pair(w_dst + kSwapWBytes + a.h0_bytes, tm_h1, full, step * kBlockK, row1);
+            if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
+        }
+    }
+    if (!alive) {
+        // Abort: give the copies in flight time to land before the pair leaves.
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < 200000ull) {}
+    }
+}
+
+template <bool kWide>
+__device__ __forceinline__ void swap_issue(const SwapLoopArgs &a, SharedControl *ctl, int32_t *status)
+{
+    int stage = 0;
+    uint32_t phase = 0;
+    bool alive = true;
+    const uint32_t idesc0 = instr_desc_bf16_m256(a.n0);
+    const uint32_t idesc1 = instr_desc_bf16_m256(kWide ? a.n1 : a.n0);
+    for (int tile = 0; tile < a.n_tiles && alive; ++tile) {
+        const uint32_t buf = kWide ? 0u : ((uint32_t)tile & 1u);                    // one accumulator when wide, else two alternate
+        const uint32_t acc_phase = (kWide ? (uint32_t)tile : ((uint32_t)tile >> 1)) & 1u;
+        if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), acc_phase ^ 1u, ctl, status)) { alive = false; break; }
+        tc_fence_after_sync();
+        const uint32_t tmem_d = a.tmem_base + buf * kSwapGroupCols;
+        for (int step = 0; step < a.k_steps; ++step) {
+            if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, ctl, status)) { alive = false; break; }
+            tc_fence_after_sync();
+            // A ragged vocabulary tile leaves stale bytes on the W tile's last rows: lanes the epilogue skips.
+            const uint32_t w_addr = a.tiles_addr + (uint32_t)stage * a.stage_bytes;
+            const uint64_t w_desc = smem_desc_k_major_sw128(w_addr);
+            const uint64_t h0_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes);
+            if (!kWide) {
+#pragma unroll
+                for (int k = 0; k < kBlockK / 16; ++k)
+                    tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h0_desc + (uint64_t)(k * 2), idesc0,
+                                     (step | k) != 0 ? 1u : 0u);
+            } else {                                             // columns 256 .. : the second group of rows, same W tile
+                const uint64_t h1_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes + a.h0_bytes);
+#pragma unroll
+                for (int k = 0; k < kBlockK / 16; ++k) {
+                    tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h0_desc + (uint64_t)(k * 2), idesc0,
+                                     (step | k) != 0 ? 1u : 0u);
+                    tc_mma_bf16_pair(a.tmem_base + kSwapGroupCols, w_desc + (uint64_t)(k * 2), h1_desc + (uint64_t)(k * 2),
+                                     idesc1, (step | k) != 0 ? 1u : 0u);
+                }
+            }
+            tc_commit_pair(smem_u32(&ctl->empty[stage]));
+            if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
+        }
+        if (alive) tc_commit_pair(smem_u32(&ctl->acc_full[buf]));
+    }
+    if (!alive) {
+        tc_commit_pair_local(smem_u32(&ctl->drain));
+        const unsigned long long t0 = global_timer_ns();
+        while (!mbar_try_wait(smem_u32(&ctl->drain), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+    }
 }
 
 __global__ void __launch_bounds__(kSwapThreads, 1)
@@ -80,7 +172,10 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     const uint32_t h1_bytes = (uint32_t)(n1 / 2) * kRowBytes;
     const uint32_t stage_bytes = (uint32_t)kSwapWBytes + h0_bytes + h1_bytes;
     SharedControl *ctl = reinterpret_cast<SharedControl *>(tiles_ptr + (size_t)n_stages * stage_bytes);
-    uint8_t *scratch = reinterpret_cast<uint8_t *>(ctl) + 512;          // kSwapScratchBytes
+    uint8_t *scratch = reinterpret_cast<uint8_t *>(ctl) + 512;          // four quadrants' scratch
+    const int warps_per_quad = swap_warps_per_quad(n_pad);
+    const int quad_scratch = swap_quad_scratch_bytes(n_pad);
+    const int epilogue_threads = 128 * warps_per_quad;                   // warps 2 .. 5, and 6 .. 9 above 256 rows
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -92,7 +187,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     const int n_tiles = split.n_tiles;
     const int k_steps = args.num_kb;
 
-    if (threadIdx.x == 0) init_pipeline_barriers(ctl, n_stages, 1, 2 * kSwapEpilogueThreads);
+    if (threadIdx.x == 0) init_pipeline_barriers(ctl, n_stages, 1, 2 * epilogue_threads);
     if (warp == 0 && lane == 0) {
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"((unsigned long long)&tm_h1) : "memory");
@@ -110,94 +205,34 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     const uint32_t tmem_base = ctl->tmem_base;
     pvf_grid_dependency_wait();
 
+    SwapLoopArgs la;
+    la.tiles_addr = tiles_addr; la.stage_bytes = stage_bytes; la.h0_bytes = h0_bytes; la.h1_bytes = h1_bytes;
+    la.tmem_base = tmem_base; la.n0 = n0; la.n1 = n1; la.n_stages = n_stages; la.n_tiles = n_tiles; la.k_steps = k_steps;
+    la.n_bufs = n_bufs; la.rank = rank;
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (one per block)
         if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            bool alive = true;
-            const int row0 = (int)rank * (n0 / 2);                                  // this block's half of each group's rows
-            const int row1 = n0 + (int)rank * (n1 / 2);
-            for (int tile = 0; tile < n_tiles && alive; ++tile) {
-                int tu0, tun;
-                split.tile(tile, &tu0, &tun);
-                const uint32_t bytes = 2u * ((uint32_t)tun * kUnitBytes + h0_bytes + h1_bytes);         // both blocks
-                const int w_row = tu0 * kPairUnit + (int)rank * tun * kUnit;                            // this block's entries
-                for (int step = 0; step < k_steps; ++step) {
-                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
-                    const uint32_t full = smem_u32(&ctl->full[stage]);
-                    const uint32_t w_dst = tiles_addr + (uint32_t)stage * stage_bytes;
-                    if (rank == 0) mbar_arrive_expect_tx(full, bytes);
-                    tma_load_2d_pair(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
-                    tma_load_2d_pair(w_dst + kSwapWBytes, &tm_h, full, step * kBlockK, row0);
-                    if (n1 > 0) tma_load_2d_pair(w_dst + kSwapWBytes + h0_bytes, &tm_h1, full, step * kBlockK, row1);
-                    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if (!alive) {
-                const unsigned long long t0 = global_timer_ns();
-                while (global_timer_ns() - t0 < 200000ull) {}
-            }
+            if (n1 == 0) swap_produce<false>(la, split, ctl, &tm_h, &tm_h1, tm_w, args.status);
+            else swap_produce<true>(la, split, ctl, &tm_h, &tm_h1, tm_w, args.status);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even block only)
         if (lane == 0 && rank == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            bool alive = true;
-            const uint32_t idesc0 = instr_desc_bf16_m256(n0);
-            const uint32_t idesc1 = instr_desc_bf16_m256(n1 > 0 ? n1 : n0);
-            for (int tile = 0; tile < n_tiles && alive; ++tile) {
-                const uint32_t buf = n_bufs == 2 ? ((uint32_t)tile & 1u) : 0u;
-                const uint32_t acc_phase = (n_bufs == 2 ? ((uint32_t)tile >> 1) : (uint32_t)tile) & 1u;
-                if (!mbar_wait(smem_u32(&ctl->acc_empty[buf]), acc_phase ^ 1u, ctl, args.status)) { alive = false; break; }
-                tc_fence_after_sync();
-                const uint32_t tmem_d = tmem_base + buf * kSwapGroupCols;
-                for (int step = 0; step < k_steps; ++step) {
-                    if (!mbar_wait(smem_u32(&ctl->full[stage]), phase, ctl, args.status)) { alive = false; break; }
-                    tc_fence_after_sync();
-                    // A ragged vocabulary tile leaves stale bytes on the W tile's last rows: lanes the epilogue skips.
-                    const uint32_t w_addr = tiles_addr + (uint32_t)stage * stage_bytes;
-                    const uint64_t w_desc = smem_desc_k_major_sw128(w_addr);
-                    const uint64_t h0_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes);
-                    const uint64_t h1_desc = smem_desc_k_major_sw128(w_addr + kSwapWBytes + h0_bytes);
-                    if (n1 == 0) {
-#pragma unroll
-                        for (int k = 0; k < kBlockK / 16; ++k)
-                            tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h0_desc + (uint64_t)(k * 2), idesc0,
-                                             (step | k) != 0 ? 1u : 0u);
-                    } else {                                     // columns 256 .. : the second group of rows, same W tile
-#pragma unroll
-                        for (int k = 0; k < kBlockK / 16; ++k) {
-                            tc_mma_bf16_pair(tmem_d, w_desc + (uint64_t)(k * 2), h0_desc + (uint64_t)(k * 2), idesc0,
-                                             (step | k) != 0 ? 1u : 0u);
-                            tc_mma_bf16_pair(tmem_base + kSwapGroupCols, w_desc + (uint64_t)(k * 2), h1_desc + (uint64_t)(k * 2),
-                                             idesc1, (step | k) != 0 ? 1u : 0u);
-                        }
-                    }
-                    tc_commit_pair(smem_u32(&ctl->empty[stage]));
-                    if (++stage == n_stages) { stage = 0; phase ^= 1u; }
-                }
-                if (alive) tc_commit_pair(smem_u32(&ctl->acc_full[buf]));
-            }
-            if (!alive) {
-                tc_commit_pair_local(smem_u32(&ctl->drain));
-                const unsigned long long t0 = global_timer_ns();
-                while (!mbar_try_wait(smem_u32(&ctl->drain), 0u) && global_timer_ns() - t0 < kWaitLimitNs) {}
-            }
+            if (n1 == 0) swap_issue<false>(la, ctl, args.status);
+            else swap_issue<true>(la, ctl, args.status);
         }
-    } else {
+    } else if (warp < 2 + 4 * warps_per_quad) {
         // ------------------------------------------------------------------ softmax epilogue (both blocks)
         const int quad = warp & 3;                                       // tensor-memory lanes quad*32 .. quad*32+31
-        const int half = (warp - 2) >> 2;                                // which of the quadrant's two warps: takes row chunks
-                                                                         // half, half + 2, half + 4, ...
+        const int half = (warp - 2) >> 2;                                // which of the quadrant's warps: takes row chunks
+                                                                         // half, half + warps_per_quad, ...
         const uint32_t lane_addr = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int n_chunks = n_pad >> 5;                                 // 32-row column groups
         const int e_thread = (int)threadIdx.x - 64;                      // 0 .. 255
-        float *turn = reinterpret_cast<float *>(scratch + quad * kSwapQuadScratchBytes + half * kSwapWarpScratchBytes);
-        float4 *fold_quad = reinterpret_cast<float4 *>(scratch + quad * kSwapQuadScratchBytes);   // [n_pad rows], after the sweep
+        float *turn = reinterpret_cast<float *>(scratch + quad * quad_scratch + half * kSwapWarpScratchBytes);
+        float4 *fold_quad = reinterpret_cast<float4 *>(scratch + quad * quad_scratch);   // [n_pad rows], after the sweep
         bool alive = true;
-        RowState st[kSwapMaxRows / 64];                                  // st[i], lane l: state of row (2 i + half) * 32 + l
+        RowState st[kSwapMaxRows / 64];                                  // st[i], lane l: state of row (warps_per_quad i + half) * 32 + l
 #pragma unroll
         for (int i = 0; i < kSwapMaxRows / 64; ++i) { st[i].m = -INFINITY; st[i].s = 0.f; st[i].t = 0.f; st[i].arg = kNoArg; }
         for (int tile = 0; tile < n_tiles && alive; ++tile) {
@@ -214,7 +249,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             if (n_real > 0) {                                                        // warp-uniform
 #pragma unroll
                 for (int i = 0; i < kSwapMaxRows / 64; ++i) {
-                    const int c = 2 * i + half;
+                    const int c = warps_per_quad * i + half;
                     if (c < n_chunks) {                                              // warp-uniform
                         uint32_t lo[16], hi[16];
                         const uint32_t col = lane_addr + buf * kSwapGroupCols + c * 32;       // column = row: group 1 starts at 256
@@ -248,22 +283,22 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
         // Fold the block's four quadrants and write the block's partial state of every row.  The row states
         // reuse the turn tiles, so every warp must have left its last tile first.  Every epilogue thread reaches
         // the barriers, aborting or not.
-        asm volatile("bar.sync 1, %0;" ::"n"(kSwapEpilogueThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"r"(epilogue_threads) : "memory");
         if (alive) {
 #pragma unroll
             for (int i = 0; i < kSwapMaxRows / 64; ++i) {
-                const int c = 2 * i + half;
+                const int c = warps_per_quad * i + half;
                 if (c < n_chunks)
                     fold_quad[c * 32 + lane] = make_float4(st[i].m, st[i].s, st[i].t, __int_as_float(st[i].arg));
             }
         }
-        asm volatile("bar.sync 1, %0;" ::"n"(kSwapEpilogueThreads) : "memory");
+        asm volatile("bar.sync 1, %0;" ::"r"(epilogue_threads) : "memory");
         if (alive && !ctl->abort_flag) {
-            for (int row = e_thread; row < args.M; row += kSwapEpilogueThreads) {
+            for (int row = e_thread; row < args.M; row += epilogue_threads) {
                 float4 acc = reinterpret_cast<const float4 *>(scratch)[row];
 #pragma unroll
                 for (int o = 1; o < 4; ++o)
-                    state_merge(acc, reinterpret_cast<const float4 *>(scratch + o * kSwapQuadScratchBytes)[row]);
+                    state_merge(acc, reinterpret_cast<const float4 *>(scratch + o * quad_scratch)[row]);
                 args.partials[(size_t)row * args.parts + 2 * q + (int)rank] = acc;
             }
         }
