@@ -42,9 +42,9 @@ NCU_TRAFFIC_PER_WAVE = {
     "pvf_score_stream_kernel": 1.04217e9,
     "pvf_score_gemm_kernel": 1.277e9,
     "pvf_score_gemm_pair_kernel": 1.0490e9,
-    "pvf_score_swap_pair_kernel": 1.0507e9,
+    "pvf_score_swap_pair_kernel": 1.0504e9,
 }
-NCU_TRAFFIC_SWAP_WIDE = 1.0579e9          # the swapped paired kernel above 256 rows (two column groups)
+NCU_TRAFFIC_SWAP_WIDE = 1.0572e9          # the swapped paired kernel above 256 rows (two column groups)
 
 
 def load_peaks():

@@ -32,6 +32,9 @@
 #ifndef PVF_SWAP_RAGGED_MAX_ROWS
 #define PVF_SWAP_RAGGED_MAX_ROWS 192   // and so do 129 .. this many rows (at most 256)
 #endif
+#ifndef PVF_SWAP_WIDE_WARPS
+#define PVF_SWAP_WIDE_WARPS 3          // epilogue warps per lane quadrant of the swapped paired kernel above 256 rows
+#endif
 #ifndef PVF_SWAP_WIDE_MAX_ROWS
 #define PVF_SWAP_WIDE_MAX_ROWS 448     // and 257 .. this many rows (at most 512; 0 = never), in two column groups
 #endif

@@ -28,8 +28,8 @@ namespace {
 // k-step (one loop serving one or two column groups) cost 17 .. 33 % of the whole launch; the two cases are
 // separate loops.
 //
-// Epilogue: eight warps, two per quadrant of 32 vocabulary lanes, each taking every other group of 32 rows
-// (columns).  A warp turns its 32 x 32 block
+// Epilogue: one warp per quadrant of 32 vocabulary lanes up to 256 rows, PVF_SWAP_WIDE_WARPS above, taking the
+// groups of 32 rows (columns) in turn.  A warp turns its 32 x 32 block
 // around through a padded shared-memory tile of its own, after which lane i holds row i's 32 logits and folds
 // them into the running state of row chunk*32 + i exactly as the GEMM kernels' epilogue does (no warp-wide
 // reductions: those serialise on their latency with one epilogue warp per scheduler).  At the end of the block's
@@ -41,14 +41,14 @@ constexpr int kSwapWBytes = kTileM * kRowBytes;                      // 16 KiB
 constexpr int kSwapGroupCols = 256;                                  // MMA N limit: columns (rows of H) per MMA
 constexpr int kSwapMaxRows = 512;                                    // two column groups fill tensor memory
 constexpr int kSwapTmemCols = 512;                                   // two accumulators of up to 256 columns, or one of up to 512
-constexpr int kSwapEpilogueWarps = 8;                                // launched; one per tensor-memory lane quadrant works on up to 256
-                                                                     // rows, two (taking alternate row chunks) above
+constexpr int kSwapEpilogueWarps = 4 * PVF_SWAP_WIDE_WARPS;          // at most; one per tensor-memory lane quadrant works on up to
+                                                                     // 256 rows, PVF_SWAP_WIDE_WARPS (taking row chunks in turn) above
 constexpr int kSwapEpilogueThreads = kSwapEpilogueWarps * 32;
 constexpr int kSwapThreads = 64 + kSwapEpilogueThreads;              // producer warp, MMA warp, epilogue warps
 constexpr int kSwapTurnPitch = 33;                                   // words per lane of a warp's 32 x 32 fp32 block (conflict-free both ways)
 constexpr int kSwapWarpScratchBytes = 32 * kSwapTurnPitch * 4;       // that block, one per epilogue warp
 // Scratch of one quadrant = its warps' blocks; at the end it holds the quadrant's row states (16 bytes per row).
-__host__ __device__ constexpr int swap_warps_per_quad(int n_pad) { return n_pad > kSwapGroupCols ? 2 : 1; }
+__host__ __device__ constexpr int swap_warps_per_quad(int n_pad) { return n_pad > kSwapGroupCols ? PVF_SWAP_WIDE_WARPS : 1; }
 __host__ __device__ constexpr int swap_quad_scratch_bytes(int n_pad) { return swap_warps_per_quad(n_pad) * kSwapWarpScratchBytes; }
 constexpr int kSwapMaxStages = 12;
 constexpr int kSwapSmemBytes = 227 * 1024;                           // everything: alignment slack, ring, control block, scratch
