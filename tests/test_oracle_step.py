@@ -308,3 +308,74 @@ def test_verify_invariants(data):
         assert extra == drafts[:ch] and len(extra) <= K
         if ch:
             assert all(tok_v[ch * nR + (drafts[q] - 1)] == tok[drafts[q]] for q in range(ch))
+
+
+# ----------------------------------------------------------------------------- C_total margins (Section 4.2, Filter 2)
+def margins_case(branch_conf, draft_r, accept, route=1):
+    """One sequence with nR remaining rows; returns c_total_margins for hand-written branch confidences."""
+    nR = len(branch_conf[0])
+    K = len(draft_r)
+    conf_v = np.concatenate([np.full(nR, 0.95)] + [np.asarray(c, dtype=np.float64) for c in branch_conf])
+    return ostep.c_total_margins(np.arange(nR, dtype=np.int32), np.array([0, nR], np.int32),
+                                 np.array([0, (1 + K) * nR], np.int32), np.array([draft_r], np.int32),
+                                 np.array([K], np.int32), np.array([route], np.uint8), conf_v,
+                                 np.array([accept], np.uint8))
+
+
+def test_c_total_margins_hand_built_three_branches():
+    # drafts at rows 1, 2, 3 of five; each branch's own draft row carries a large value that must be left out:
+    #   C_1 = 0.5 + 0.6 + 0.4 + 0.4    = 1.9       (row 1 = 9.0 left out)
+    #   C_2 = 0.5 + 0.6 + 0.6 + 0.6    = 2.3       (row 2 = 7.0 left out)
+    #   C_3 = 0.5 + 0.6 + 0.6 + 0.6005 = 2.3005    (row 3 = 5.0 left out)
+    bc = [[0.5, 9.0, 0.6, 0.4, 0.4], [0.5, 0.6, 7.0, 0.6, 0.6], [0.5, 0.6, 0.6, 5.0, 0.6005]]
+    m = margins_case(bc, [1, 2, 3], [1, 1, 1])
+    assert m.shape == (1,) and abs(m[0] - 0.0005) < 1e-12
+    # only accepted branches count: without branch 3 the closest pair is C_2 - C_1 = 0.4
+    assert abs(margins_case(bc, [1, 2, 3], [1, 1, 0])[0] - 0.4) < 1e-12
+    assert abs(margins_case(bc, [1, 2, 3], [1, 0, 1])[0] - 0.4005) < 1e-12
+    # the result does not depend on the order the branches come in
+    assert abs(margins_case([bc[2], bc[0], bc[1]], [3, 1, 2], [1, 1, 1])[0] - 0.0005) < 1e-12
+
+
+def test_c_total_margins_is_inf_without_two_accepted_planning_branches():
+    bc = [[0.5, 9.0, 0.6], [0.5, 0.6, 7.0]]
+    assert np.isinf(margins_case(bc, [1, 2], [1, 0])[0])
+    assert np.isinf(margins_case(bc, [1, 2], [0, 0])[0])
+    assert np.isinf(margins_case(bc, [1, 2], [1, 1], route=2)[0])        # AR route: Filter 2 does not apply
+    assert np.isinf(margins_case(bc, [1, 2], [1, 1], route=0)[0])
+    assert abs(margins_case(bc, [1, 2], [1, 1])[0] - 0.0) < 1e-12        # C_1 = C_2 = 1.1: an exact tie
+
+
+def test_c_total_margins_agree_with_verifys_choice():
+    # verify picks the accepted branch with the largest C_total; margins computed independently must rank the
+    # same branch on top whenever the margin is clear, on random cases of several sequences
+    rng = np.random.default_rng(5)
+    for _ in range(40):
+        n_seq, K = 3, 3
+        nRs = rng.integers(3, 7, n_seq)
+        seg = np.concatenate([[0], np.cumsum(nRs)]).astype(np.int32)
+        M = int(seg[-1])
+        pos = np.concatenate([np.arange(n) for n in nRs]).astype(np.int32)
+        rem, rem_off = np.arange(M, dtype=np.int32), seg.copy()
+        dr = np.stack([seg[b] + np.sort(rng.permutation(nRs[b])[:K]) for b in range(n_seq)]).astype(np.int32)
+        nd = np.full(n_seq, K, np.int32)
+        v_off = np.concatenate([[0], np.cumsum((1 + K) * nRs)]).astype(np.int32)
+        tok = np.arange(M, dtype=np.int32)
+        tok_v = np.concatenate([np.tile(tok[seg[b]:seg[b + 1]], 1 + K) for b in range(n_seq)]).astype(np.int32)
+        conf_v = rng.uniform(0.0, 1.0, int(v_off[-1]))
+        for b in range(n_seq):
+            conf_v[v_off[b]] = 0.99                                       # a non-empty impact set everywhere
+        route = np.ones(n_seq, np.uint8)
+        r = ostep.verify(tok, np.zeros(M, np.uint8), seg, pos, rem, rem_off, v_off, dr, nd, route, tok_v, conf_v, 0.9, K)
+        assert r["accept"].all()
+        m = ostep.c_total_margins(rem, rem_off, v_off, dr, nd, route, conf_v, r["accept"])
+        for b in range(n_seq):
+            nR = int(nRs[b])
+            cs = []
+            for j in range(1, K + 1):
+                blk = conf_v[v_off[b] + j * nR: v_off[b] + (j + 1) * nR].copy()
+                blk[dr[b, j - 1] - seg[b]] = 0.0
+                cs.append(blk.sum())
+            srt = np.sort(cs)
+            assert abs(m[b] - np.min(np.diff(srt))) < 1e-12
+            assert int(r["choice"][b]) == int(np.argmax(cs)) + 1
