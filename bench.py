@@ -144,6 +144,14 @@ def whole_job_value(rows_per_rank: int, steps: int, ms: float, world: int) -> fl
 
 
 # ------------------------------------------------------------------------------------ reference arm
+def workload_config(name, st, **more):
+    """The `config` object of a line: both arms print the same `workload` string."""
+    cfg = dict(workload=name, generator=st.name, vocab=st.vocab, hidden=st.hidden, n_seq=st.n_seq, draft_rows=st.n_rows,
+               budget=int(st.params["budget"]), tau_high=st.params["tau_high"])
+    cfg.update(more)
+    return cfg
+
+
 def run_reference(args):
     """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -181,28 +189,82 @@ def run_reference(args):
     line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=1e3 * dt / args.steps, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
-                config=dict(workload=args.workload, vocab=st.vocab, hidden=st.hidden, rows_per_step=rows),
+                config=workload_config(args.workload, st, rows_per_step=rows),
                 cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------ our arm
-def run_ours(args):
+EVENT_EVERY = 8            # the projection kernel is timed on every 8th step of the timed region
+MAX_EVENT_PAIRS = 4096     # events created before the timed region
+MAX_REPEATS = 2000
+
+
+def gpu_id_of(dev, local_rank):
     import torch
-    from paper_2601_12247_b200 import binding, synth
+    props = torch.cuda.get_device_properties(dev)
+    if hasattr(props, "uuid"):
+        return "GPU-" + str(props.uuid)
+    visible = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    return visible.split(",")[local_rank] if visible else str(local_rank)
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group(backend="nccl", device_id=dev)
-    peaks = load_peaks()
 
-    st = make_workload(args.workload, synth)
+def roofline_of(pairs, ctx, V, D, peaks, sm_mhz, event_every):
+    """Roofline object of the projection launches timed by `pairs` = [(start event, stop event, rows)].
+
+    achieved = algorithmic bytes (or flops) of those launches / their summed CUDA-event durations; the bound is the
+    slower of the two roofline times.  A tensor-bound mix reports its fraction of the burst bf16 peak (`frac`) and of
+    the sustained one (`frac_sustained`)."""
+    durs = [(a.elapsed_time(b), r) for a, b, r in pairs]
+    gemm_ms = sum(d for d, _ in durs)
+    n = len(durs)
+    alg_bytes = sum(2.0 * V * D + 2.0 * r * D + 13.0 * r + V / 8.0 for _, r in durs)
+    alg_flops = sum(2.0 * r * V * D for _, r in durs)
+    t = gemm_ms * 1e-3
+    if alg_bytes / (peaks["hbm_gbs"] * 1e9) >= alg_flops / (peaks["bf16_tflops"] * 1e12):
+        roof = dict(bound="hbm", achieved=alg_bytes / t / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["peak_source"] = peaks["source"] + " (copy bandwidth)"
+    else:
+        roof = dict(bound="tensor", achieved=alg_flops / t / 1e12, peak=peaks["bf16_tflops"], unit="TFLOP/s")
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["peak_sustained"] = peaks["bf16_tflops_sustained"]
+        roof["frac_sustained"] = roof["achieved"] / peaks["bf16_tflops_sustained"]
+        roof["peak_source"] = peaks["source"] + " (cuBLAS bf16: burst; sustained beside it)"
+
+    def launch_traffic(rows):
+        name = ctx.score_kernel_name(rows)
+        per_wave = NCU_TRAFFIC_SWAP_WIDE if (name == "pvf_score_swap_pair_kernel" and rows > 256) else NCU_TRAFFIC_PER_WAVE.get(name)
+        return None if per_wave is None else per_wave * ctx.score_plan(rows)["waves"]
+    per_launch = [launch_traffic(r) for _, r in durs]
+    traffic = sum(per_launch) / n if per_launch and all(x is not None for x in per_launch) else None
+    by_rows = {}
+    for d, r in durs:
+        by_rows.setdefault(r, []).append(d)
+    per_rows = []
+    for r in sorted(by_rows):
+        us = 1e3 * float(np.mean(by_rows[r]))
+        item = dict(rows=r, kernel=ctx.score_kernel_name(r), launches=len(by_rows[r]), avg_launch_us=us,
+                    tflops=2.0 * r * V * D / (us * 1e-6) / 1e12,
+                    gbs=(2.0 * V * D + 2.0 * r * D + 13.0 * r + V / 8.0) / (us * 1e-6) / 1e9)
+        if sm_mhz:
+            item["sm_cycles_per_launch"] = us * sm_mhz
+        per_rows.append(item)
+    roof.update(traffic=traffic, kernel="+".join(sorted({ctx.score_kernel_name(r) for _, r in durs})), launches=n,
+                timed_every_nth_step=event_every, avg_launch_us=1e3 * gemm_ms / max(n, 1),
+                algorithmic_bytes_per_launch=alg_bytes / max(n, 1), algorithmic_flops_per_launch=alg_flops / max(n, 1),
+                sm_mhz_median=sm_mhz, sm_cycles_per_launch=(1e3 * gemm_ms / max(n, 1)) * sm_mhz if sm_mhz else None,
+                per_row_count=per_rows)
+    return roof
+
+
+def run_workload(name, synth, binding, dev, world, rank, local_rank, peaks, steps, warmup, event_every, min_seconds,
+                 want_e2e, want_graph, cpu_rows):
+    """Times one workload: `steps` steps per timed block (CUDA events around the block, barrier and synchronise on
+    both sides), blocks repeated until `min_seconds` have passed; the reported step time is the median block's."""
+    import torch
+    st = make_workload(name, synth)
     p = st.params
     M, V, D = st.n_rows, st.vocab, st.hidden
     K = int(p["budget"])
@@ -239,13 +301,11 @@ def run_ours(args):
     o_ver = dict(accept=torch.empty((st.n_seq, K), dtype=torch.uint8, device=dev),
                  choice=torch.empty(st.n_seq, dtype=torch.int32, device=dev),
                  final_commit=torch.empty(M, dtype=torch.uint8, device=dev))
-    # The projection kernel is timed on every `event_every`-th step of the timed region: events around a launch
-    # cost the overlap of its set-up with the previous kernel, so timing all of them would slow the step it measures.
-    event_every = 8 if args.steps >= 64 else 1
-    n_event_steps = (args.steps + event_every - 1) // event_every
+    # Events around the projection launches cost the overlap of a launch's set-up with the previous kernel, so only
+    # every `event_every`-th step of the timed region carries them (every step where the kernels run for milliseconds).
     ev_pairs = []
     ev_pool = []
-    for _ in range(2 * n_event_steps):             # created (and first recorded) outside the timed region
+    for _ in range(MAX_EVENT_PAIRS):               # created (and first recorded) outside the timed region
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(); b.record()
         ev_pool.append((a, b))
@@ -253,6 +313,7 @@ def run_ours(args):
 
     def step(h_dev, hv_dev, timed_events=False):
         launches = 0
+        timed_events = timed_events and len(ev_pool) >= 2
         if not timed_events:
             ctx.set_score_events(None, None)
         if timed_events:
@@ -276,34 +337,39 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     # ---------------- device-resident timing
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         step(h, hv)
     barrier()
-    props = torch.cuda.get_device_properties(dev)
-    if hasattr(props, "uuid"):
-        gpu_id = "GPU-" + str(props.uuid)
-    else:
-        visible = os.environ.get("CUDA_VISIBLE_DEVICES", "")
-        gpu_id = visible.split(",")[local_rank] if visible else str(local_rank)
-    sampler = ClockSampler(gpu_id)
+    sampler = ClockSampler(gpu_id_of(dev, local_rank))
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches = 0
-    e0.record()
-    for i in range(args.steps):
-        launches += step(h, hv, timed_events=(i % event_every == 0))
-    e1.record()
-    barrier()
+    block_ms, launches, n_steps_run = [], 0, 0
+    t_wall = time.perf_counter()
+    while True:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            n = step(h, hv, timed_events=(n_steps_run % event_every == 0))
+            n_steps_run += 1
+            if not block_ms:
+                launches += n                      # kernels launched inside one timed block of `steps` steps
+        e1.record()
+        barrier()
+        block_ms.append(max_over_ranks(e0.elapsed_time(e1), dev))
+        # every rank takes the same decision: the block times are already the maximum over ranks
+        enough = sum(block_ms) * 1e-3 >= min_seconds or time.perf_counter() - t_wall >= 4.0 * max(min_seconds, 0.5)
+        if enough or len(block_ms) >= MAX_REPEATS:
+            break
     clocks = sampler.stop()
     ctx.set_score_events(None, None)
-    ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    ms = float(np.median(block_ms))
     status = ctx.last_status()
-    value = whole_job_value(M, args.steps, ms, world)
+    value = whole_job_value(M, steps, ms, world)
+    roof = roofline_of(ev_pairs, ctx, V, D, peaks, clocks.get("sm_mhz"), event_every)
 
     # ---------------- the same step captured once in a CUDA graph and replayed (no per-launch host work, no events
     # between the kernels): reported beside the main number
     graph_replay = None
-    if not args.no_graph:
+    if want_graph:
         try:
             side = torch.cuda.Stream(device=dev)
             side.wait_stream(torch.cuda.current_stream())
@@ -317,124 +383,181 @@ def run_ours(args):
             for _ in range(3):
                 graph.replay()
             barrier()
+            n_graph = max(steps, 200)
             g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             g0.record()
-            for _ in range(args.steps):
+            for _ in range(n_graph):
                 graph.replay()
             g1.record()
             barrier()
             ms_graph = max_over_ranks(g0.elapsed_time(g1), dev)
-            graph_replay = dict(value=whole_job_value(M, args.steps, ms_graph, world), unit=UNIT, ms_per_step=ms_graph / args.steps)
+            graph_replay = dict(value=whole_job_value(M, n_graph, ms_graph, world), unit=UNIT, steps=n_graph,
+                                ms_per_step=ms_graph / n_graph)
         except RuntimeError as exc:                    # capture not possible here: report it, the main number stands
             graph_replay = dict(unavailable=str(exc)[:200])
 
-    # roofline of the dominant kernel (the score GEMM), from the events recorded in the timed region
-    gemm_ms = sum(a.elapsed_time(b) for a, b, _ in ev_pairs)
-    rows_scored = sum(r for _, _, r in ev_pairs)
-    n_gemm = len(ev_pairs)
-    alg_bytes = sum(2.0 * V * D + 2.0 * r * D + 13.0 * r + V / 8.0 for _, _, r in ev_pairs)
-    alg_flops = sum(2.0 * r * V * D for _, _, r in ev_pairs)
-    t_gemm = gemm_ms * 1e-3
-    hbm_time = alg_bytes / (peaks["hbm_gbs"] * 1e9)
-    tc_time = alg_flops / (peaks["bf16_tflops_sustained"] * 1e12)
-    if hbm_time >= tc_time:
-        roof = dict(bound="hbm", achieved=alg_bytes / t_gemm / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
-    else:
-        roof = dict(bound="tensor", achieved=alg_flops / t_gemm / 1e12, peak=peaks["bf16_tflops_sustained"], unit="TFLOP/s")
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    kernels = sorted({ctx.score_kernel_name(r) for _, _, r in ev_pairs})
-    def launch_traffic(rows):
-        name = ctx.score_kernel_name(rows)
-        return NCU_TRAFFIC_SWAP_WIDE if (name == "pvf_score_swap_pair_kernel" and rows > 256) else NCU_TRAFFIC_PER_WAVE.get(name)
-    per_launch = [launch_traffic(r) for _, _, r in ev_pairs]
-    if per_launch and all(t is not None for t in per_launch):       # average launch of the timed mix
-        traffic = sum(t * ctx.score_plan(r)["waves"] for t, (_, _, r) in zip(per_launch, ev_pairs)) / n_gemm
-    else:
-        traffic = None
-    roof.update(traffic=traffic, kernel="+".join(kernels), launches=n_gemm, timed_every_nth_step=event_every, avg_launch_us=1e3 * gemm_ms / max(n_gemm, 1),
-                algorithmic_bytes_per_launch=alg_bytes / max(n_gemm, 1), peak_source=peaks["source"] +
-                (" (sustained bf16)" if roof["bound"] == "tensor" else " (copy bandwidth)"))
-
     # ---------------- end to end: the host-buffer C entry points (inputs in pinned host memory, every
     # result copied back to host memory, stream synchronised inside each call)
-    n_e2e = max(3, min(args.steps, 200))
-    ctx.attach_host_staging()
-    hb = binding.host_buffers(M, st.n_seq, K, Mv)
-    seg_h = torch.from_numpy(np.ascontiguousarray(st.seg_off, dtype=np.int32)).pin_memory()
-    pos_h = torch.from_numpy(np.ascontiguousarray(st.row_pos, dtype=np.int32)).pin_memory()
-    act_h = torch.from_numpy(np.ascontiguousarray(st.active)).pin_memory()
+    e2e = None
+    if want_e2e:
+        n_e2e = max(3, min(steps, 200))
+        ctx.attach_host_staging()
+        hb = binding.host_buffers(M, st.n_seq, K, Mv)
+        seg_h = torch.from_numpy(np.ascontiguousarray(st.seg_off, dtype=np.int32)).pin_memory()
+        pos_h = torch.from_numpy(np.ascontiguousarray(st.row_pos, dtype=np.int32)).pin_memory()
+        act_h = torch.from_numpy(np.ascontiguousarray(st.active)).pin_memory()
 
-    def e2e_step():
-        ctx.draft_step_host(prm, h_host, seg_h, pos_h, act_h, hb)
-        ctx.verify_step_host(prm, hv_host, hb)
+        def e2e_step():
+            ctx.draft_step_host(prm, h_host, seg_h, pos_h, act_h, hb)
+            ctx.verify_step_host(prm, hv_host, hb)
 
-    for _ in range(3):
-        e2e_step()
-    if int(hb["v_off"][-1]) != Mv:
-        raise SystemExit("host-buffer step laid out %d verification rows, expected %d" % (int(hb["v_off"][-1]), Mv))
-    barrier()
-    e0.record()
-    for _ in range(n_e2e):
-        e2e_step()
-    e1.record()
-    barrier()
-    ms_e2e = max_over_ranks(e0.elapsed_time(e1), dev)
-    h2d = int(h_host.numel() * 2 + (hv_host.numel() * 2 if Mv else 0) + seg_h.numel() * 4 + pos_h.numel() * 4 + act_h.numel())
-    d2h_keys_draft = ("tok", "conf", "ent", "in_plan", "commit", "draft_rows", "n_drafts", "route", "rem_off", "v_off")
-    d2h = int(sum(hb[k].numel() * hb[k].element_size() for k in d2h_keys_draft) + M * 4        # rem_rows: M entries
-              + Mv * 8 + hb["accept"].numel() + hb["choice"].numel() * 4 + M)
-    e2e = dict(value=whole_job_value(M, n_e2e, ms_e2e, world), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
-               steps=n_e2e, ms_per_step=ms_e2e / n_e2e, api="pvf_draft_step_host + pvf_verify_step_host")
+        for _ in range(3):
+            e2e_step()
+        if int(hb["v_off"][-1]) != Mv:
+            raise SystemExit("host-buffer step laid out %d verification rows, expected %d" % (int(hb["v_off"][-1]), Mv))
+        e2e_blocks = []
+        t_wall = time.perf_counter()
+        while True:
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n_e2e):
+                e2e_step()
+            e1.record()
+            barrier()
+            e2e_blocks.append(max_over_ranks(e0.elapsed_time(e1), dev))
+            if sum(e2e_blocks) * 1e-3 >= min(min_seconds, 1.0) or time.perf_counter() - t_wall >= 4.0 or len(e2e_blocks) >= MAX_REPEATS:
+                break
+        ms_e2e = float(np.median(e2e_blocks))
+        h2d = int(h_host.numel() * 2 + (hv_host.numel() * 2 if Mv else 0) + seg_h.numel() * 4 + pos_h.numel() * 4 + act_h.numel())
+        d2h_keys_draft = ("tok", "conf", "ent", "in_plan", "commit", "draft_rows", "n_drafts", "route", "rem_off", "v_off")
+        d2h = int(sum(hb[k].numel() * hb[k].element_size() for k in d2h_keys_draft) + M * 4        # rem_rows: M entries
+                  + Mv * 8 + hb["accept"].numel() + hb["choice"].numel() * 4 + M)
+        e2e = dict(value=whole_job_value(M, n_e2e, ms_e2e, world), unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                   steps=n_e2e, repeats=len(e2e_blocks), ms_per_step=ms_e2e / n_e2e,
+                   api="pvf_draft_step_host + pvf_verify_step_host")
 
     # ---------------- CPU baseline: the oracle on the same step (rank 0, single-GPU runs only)
     cpu = parity = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and cpu_rows > 0:
         from oracle import score as oscore
         from oracle import step as ostep
-        rows = min(M, args.cpu_rows)
-        rows_v = min(Mv, args.cpu_rows)
+        rows = min(M, cpu_rows)
+        rows_v = min(Mv, cpu_rows)
+        # an evenly spread sample when the pass is larger than the sample (the first rows belong to one sequence)
+        pick = np.arange(rows) if rows == M else np.unique(np.linspace(0, M - 1, rows).astype(np.int64))
+        pick_v = np.arange(rows_v) if rows_v == Mv else np.unique(np.linspace(0, Mv - 1, rows_v).astype(np.int64))
+        rows, rows_v = len(pick), len(pick_v)
         t0 = time.perf_counter()
-        osc = oscore.score(st.w_bits, st.h_bits[:rows], st.plan_ids)
+        osc = oscore.score(st.w_bits, st.h_bits[pick], st.plan_ids)
         if rows == M:
             ocm = ostep.commit(osc["conf"], osc["tok"], st.seg_off, st.row_pos, st.active, p["tau_high"])
             ostep.select_drafts(osc["conf"], osc["tok"], osc["in_plan"], ocm["commit"], st.seg_off, st.row_pos,
                                 st.active, p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], K)
-        oscv = oscore.score(st.w_bits, vp.hv_bits[:rows_v], st.plan_ids) if rows_v else None
+        oscv = oscore.score(st.w_bits, vp.hv_bits[pick_v], st.plan_ids) if rows_v else None
         dt = time.perf_counter() - t0
         # parity of the step just timed against the same oracle results (outside the timed regions)
         g = {k: v.cpu().numpy() for k, v in o_sc.items()}
         near = osc["gap"] < 1e-3
-        parity = dict(rows=rows, max_conf_err=float(np.max(np.abs(g["conf"][:rows] - osc["conf"]))),
-                      max_ent_err=float(np.max(np.abs(g["ent"][:rows] - osc["ent"]))),
+        parity = dict(rows=rows, max_conf_err=float(np.max(np.abs(g["conf"][pick] - osc["conf"]))),
+                      max_ent_err=float(np.max(np.abs(g["ent"][pick] - osc["ent"]))),
                       near_tie_rows=int(near.sum()),
-                      token_mismatches_outside_near_ties=int((g["tok"][:rows][~near] != osc["tok"][~near]).sum()))
+                      token_mismatches_outside_near_ties=int((g["tok"][pick][~near] != osc["tok"][~near]).sum()))
         if oscv is not None:
             gv = {k: v.cpu().numpy() for k, v in o_scv.items()}
             nearv = oscv["gap"] < 1e-3
-            parity.update(verify_rows=rows_v, max_conf_err_verify=float(np.max(np.abs(gv["conf"][:rows_v] - oscv["conf"]))),
+            parity.update(verify_rows=rows_v, max_conf_err_verify=float(np.max(np.abs(gv["conf"][pick_v] - oscv["conf"]))),
                           near_tie_rows_verify=int(nearv.sum()),
-                          token_mismatches_outside_near_ties_verify=int((gv["tok"][:rows_v][~nearv] != oscv["tok"][~nearv]).sum()))
+                          token_mismatches_outside_near_ties_verify=int((gv["tok"][pick_v][~nearv] != oscv["tok"][~nearv]).sum()))
         frac = (rows + rows_v) / float(M + Mv)
         cpu = dict(value=M * frac / dt, unit=UNIT, cores=oscore.threads(), kind="oracle", seconds=dt,
                    sample="%d of %d draft-pass rows and %d of %d verification-pass rows of the same step, fp64 score%s"
                           % (rows, M, rows_v, Mv, " + commit + draft selection" if rows == M else ""))
 
-    if rank == 0:
-        geo = ctx.score_plan(M)
-        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
-                    ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
-                    data="synthetic",
-                    config=dict(workload=args.workload + " (" + st.name + ")", vocab=V, hidden=D, n_seq=st.n_seq,
-                                draft_rows=M, verify_rows=Mv, budget=K, tau_high=p["tau_high"],
-                                step="score+commit+select+score(verify)+verify",
-                                l2="inputs larger than L2: the 1.04 GB weight matrix is streamed from HBM every score call",
-                                parallelism="replicas" if world > 1 else "single GPU", score_geometry=geo),
-                    clocks=dict(sm_mhz=clocks.get("sm_mhz"), sm_max_mhz=clocks.get("sm_max_mhz"),
-                                reasons=clocks.get("reasons", []), samples=clocks.get("samples", 0),
-                                power_w_max=clocks.get("power_w_max")),
-                    e2e=e2e, gpu_launches=launches, roofline=roof, cpu_baseline=cpu, parity=parity, graph_replay=graph_replay, status=status)
-        print(json.dumps(line))
+    geo = ctx.score_plan(M)
+    res = dict(st=st, M=M, Mv=Mv, K=K, value=value, ms_per_step=ms / steps, repeats=len(block_ms),
+               block_ms_min=float(min(block_ms)), block_ms_max=float(max(block_ms)), launches=launches, roofline=roof,
+               clocks=dict(sm_mhz=clocks.get("sm_mhz"), sm_max_mhz=clocks.get("sm_max_mhz"), reasons=clocks.get("reasons", []),
+                           samples=clocks.get("samples", 0), power_w_max=clocks.get("power_w_max")),
+               e2e=e2e, cpu_baseline=cpu, parity=parity, graph_replay=graph_replay, status=status, geometry=geo)
     ctx.close()
+    del ctx, h, hv
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_decode_loop(synth, binding, dev):
+    """BASELINE config 4: the synthetic decode loop (Algorithm 1) at batch 32, 256 tokens, blocks of 32, budget 4,
+    PVF against confidence-threshold-only decoding (budget 0) on the same targets."""
+    from paper_2601_12247_b200 import decode_loop
+    V, D, B, L, S, K, seed = synth.LLADA_VOCAB, synth.LLADA_HIDDEN, 32, 256, 32, 4, 1004
+    mask = V - 128
+    w_bits = synth.make_w(seed, V, D)
+    plan = synth.make_plan_ids(seed, V, 2048)
+    targets = synth.loop_targets(seed, V, B, L, plan, 0.0, avoid=mask)
+    ctx = binding.Context(binding.bf16_from_bits(w_bits, dev), plan, B * S * (2 + K), B, K)
+    p = dict(tau_high=0.9, budget=K, **synth.DEFAULT_BAND)
+    out = dict(workload="cfg4 (decode loop)", n_seq=B, gen_len=L, block=S, budget=K, tau_high=0.9, data="synthetic",
+               note="a step is one batched forward (draft pass + verification branches); hidden states re-drawn per step on "
+                    "the host; kernel_ms_per_step = CUDA-event time of the library's kernels only")
+    for key, budget in (("pvf", K), ("threshold_only", 0)):
+        r = decode_loop.decode(ctx, w_bits, targets, seed, L, S, dict(p, budget=budget), mask)
+        out[key] = dict(steps=r["steps"], mean_steps_per_sequence=float(r["steps_per_seq"].mean()),
+                        tokens_per_forward=r["tokens_per_forward"], scored_rows=r["scored_rows"],
+                        kernel_ms_per_step=r["kernel_ms_per_step"], kernel_ms_total=r["kernel_ms_total"],
+                        all_committed=bool((r["y"] != mask).all()), status=r["status"])
+    out["steps_ratio"] = out["threshold_only"]["steps"] / max(out["pvf"]["steps"], 1)
+    ctx.close()
+    return out
+
+
+def run_ours(args):
+    import torch
+    from paper_2601_12247_b200 import binding, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group(backend="nccl", device_id=dev)
+    peaks = load_peaks()
+    heavy = args.workload in ("cfg3", "cfg3s")
+    r = run_workload(args.workload, synth, binding, dev, world, rank, local_rank, peaks, args.steps, args.warmup,
+                     1 if heavy else EVENT_EVERY, args.min_seconds, True, not args.no_graph,
+                     0 if args.no_cpu_baseline else args.cpu_rows)
+    st = r["st"]
+    line = dict(metric=METRIC, value=r["value"], unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                ms_per_step=r["ms_per_step"], higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic",
+                config=workload_config(args.workload, st, verify_rows=r["Mv"], step="score+commit+select+score(verify)+verify",
+                                       l2="inputs larger than L2: the 1.04 GB weight matrix is streamed from HBM every score call",
+                                       parallelism="replicas" if world > 1 else "single GPU", score_geometry=r["geometry"],
+                                       timing="median of %d timed blocks of %d steps (blocks repeated for >= %.1f s; "
+                                              "fastest %.4f, slowest %.4f ms per step)"
+                                              % (r["repeats"], args.steps, args.min_seconds, r["block_ms_min"] / args.steps,
+                                                 r["block_ms_max"] / args.steps)),
+                repeats=r["repeats"], clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["launches"], roofline=r["roofline"],
+                cpu_baseline=r["cpu_baseline"], parity=r["parity"], graph_replay=r["graph_replay"], status=r["status"])
+
+    # ---------------- beside the headline (single-GPU default run): the tensor-bound regime (BASELINE config 3) and
+    # the decode loop (BASELINE config 4), measured in the same process
+    if world == 1 and args.workload == "cfg1a":
+        if not args.no_tensor_regime:
+            steps3 = 4
+            t = run_workload("cfg3", synth, binding, dev, world, rank, local_rank, peaks, steps3, 3, 1, args.min_seconds,
+                             False, False, 0 if args.no_cpu_baseline else 8)
+            line["tensor_regime"] = dict(workload="cfg3", generator=t["st"].name, draft_rows=t["M"], verify_rows=t["Mv"],
+                                         steps=steps3, repeats=t["repeats"], ms_per_step=t["ms_per_step"], value=t["value"],
+                                         unit=UNIT, gpu_launches=t["launches"], roofline=t["roofline"], clocks=t["clocks"],
+                                         parity=t["parity"], cpu_baseline=t["cpu_baseline"], status=t["status"],
+                                         score_geometry=t["geometry"])
+        if not args.no_decode_loop:
+            line["decode_loop"] = run_decode_loop(synth, binding, dev)
+    if rank == 0:
+        print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
@@ -443,13 +566,17 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=200, help="steps per timed block")
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg1a", choices=["cfg1a", "cfg1b", "cfg2", "cfg2w", "cfg3", "cfg3s", "dream1a", "dream1b"])
+    ap.add_argument("--min-seconds", type=float, default=2.0,
+                    help="the timed block of --steps steps is repeated until this much GPU time has passed; the median block is reported")
     ap.add_argument("--cpu-rows", type=int, default=256, help="rows per pass the CPU baseline scores")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay of the step")
+    ap.add_argument("--no-tensor-regime", action="store_true", help="skip the config-3 object of the default run")
+    ap.add_argument("--no-decode-loop", action="store_true", help="skip the config-4 object of the default run")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

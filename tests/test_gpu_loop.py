@@ -163,3 +163,74 @@ def test_calibration_trajectory_matches_oracle():
         assert np.array_equal(st["sum_a"], want["stats"]["sum_a"])
         assert np.max(np.abs(st["sum_vig_q32"] / 2.0 ** 32 - want["stats"]["sum_vig"])) <= 2e-3 * max(1, want["n_events"])
     ctx.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("q_plan", [0.0, 0.5])
+def test_loop_config4_full_size(q_plan):
+    # Config 4 at its stated size (Algorithm 1): LLaDA-shaped head, 32 sequences, 256 tokens, blocks of 32, budget 4,
+    # forced progress.  Per step: sampled draft and verification rows against the oracle one by one, and every
+    # decision of the step against the oracle's rules fed the GPU's own fp32 outputs.  At the end: no mask left,
+    # committed tokens never changed, and PVF needs no more forwards than threshold-only decoding (K = 0).
+    V, D, B, L, S, K, seed = synth.LLADA_VOCAB, synth.LLADA_HIDDEN, 32, 256, 32, 4, 1004
+    mask = V - 128
+    w = synth.make_w(seed, V, D)
+    plan = synth.make_plan_ids(seed, V, 2048)
+    tg = synth.loop_targets(seed, V, B, L, plan, q_plan, avoid=mask)
+    p = dict(tau_high=0.9, budget=K, **synth.DEFAULT_BAND)
+    ctx = make_ctx(w, plan, B * S * (2 + K), B, K)
+    state = dict(prev=np.full((B, L), mask, np.int32), rows=0, rows_v=0, routes=np.zeros(3, np.int64), checked=0, checked_v=0)
+
+    def on_step(s, d):
+        from oracle import step as ostep
+        pos, seg = d["positions"], d["seg_off"]
+        n = len(pos)
+        act = np.ones(n, np.uint8)
+        g_sc = to_np(d["score"])
+        assert n <= B * S and np.all(np.diff(seg) <= S)
+        if n and (s < 4 or s % 4 == 0):                                    # sampled rows against the oracle
+            rows = np.unique(np.array([0, n // 2, n - 1]))
+            check_score(g_sc, oscore.score(w, d["h_bits"][rows], plan), V, plan, rows=rows)
+            state["checked"] += len(rows)
+        conf64 = g_sc["conf"].astype(np.float64)
+        ocm = ostep.commit(conf64, g_sc["tok"], seg, pos, act, p["tau_high"], force_progress=True)
+        assert np.array_equal(to_np(d["commit"])["commit"], ocm["commit"])
+        osel = ostep.select_drafts(conf64, g_sc["tok"], g_sc["in_plan"], ocm["commit"], seg, pos, act,
+                                   p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], K)
+        gs = to_np(d["select"])
+        for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+            assert np.array_equal(gs[k], osel[k]), (s, k)
+        state["routes"] += np.bincount(osel["route"], minlength=3)
+        Mv = int(osel["v_off"][-1])
+        g_scv = to_np(d["score_v"])
+        if Mv and (s < 4 or s % 4 == 0):
+            rows = np.unique(np.array([0, Mv // 2, Mv - 1]))
+            check_score(g_scv, oscore.score(w, d["hv_bits"][rows], plan), V, plan, rows=rows)
+            state["checked_v"] += len(rows)
+        over = ostep.verify(g_sc["tok"], ocm["commit"], seg, pos, osel["rem_rows"], osel["rem_off"], osel["v_off"],
+                            osel["draft_rows"], osel["n_drafts"], osel["route"], g_scv["tok"][:max(Mv, 0)],
+                            g_scv["conf"][:max(Mv, 0)].astype(np.float64), p["tau_high"], K)
+        gv = to_np(d["verify"])
+        for k in ("accept", "choice", "final_commit"):
+            assert np.array_equal(gv[k], over[k]), (s, k)
+        # the canvas: exactly the final commits are written, with the draft pass's tokens; nothing else changes
+        want_y = state["prev"].copy()
+        fin = over["final_commit"].astype(bool)
+        want_y[d["seq_ids"][fin], pos[fin]] = g_sc["tok"][fin]
+        assert np.array_equal(d["y"], want_y)
+        assert fin.sum() >= (np.diff(seg) > 0).sum()                       # forced progress: every live sequence moves
+        state["prev"] = d["y"]
+        state["rows"] += n
+        state["rows_v"] += Mv
+
+    got = decode_loop.decode(ctx, w, tg, seed, L, S, p, mask, on_step=on_step)
+    assert got["status"] == 0 and not (got["y"] == mask).any()
+    assert state["checked"] >= 9 and got["scored_rows"] == state["rows"] + state["rows_v"]
+    assert state["routes"][1] + state["routes"][2] > 0 and state["rows_v"] > 0
+    if q_plan > 0:
+        assert state["routes"][1] > 0 and state["checked_v"] > 0         # the planning route was taken
+    base = decode_loop.decode(ctx, w, tg, seed, L, S, dict(p, budget=0), mask)
+    assert base["status"] == 0 and not (base["y"] == mask).any()
+    assert got["steps"] <= base["steps"] and got["tokens_per_forward"] >= base["tokens_per_forward"] - 1e-9
+    assert 1.0 <= base["tokens_per_forward"] <= S and got["steps_per_seq"].min() >= L // S
+    ctx.close()

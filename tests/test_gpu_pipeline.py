@@ -307,3 +307,85 @@ def test_config3_large_batch_sampled(llada):
         assert np.array_equal(gs["draft_rows"][b], want_rows)
         assert gs["route"][b] == osel1["route"][0] and gs["n_drafts"][b] == osel1["n_drafts"][0]
         assert gs["rem_off"][b + 1] - gs["rem_off"][b] == osel1["rem_off"][1]
+
+
+def torch_fp64_reference(w_head, h_dev, chunk=1024):
+    """Every row of a launch against a second reference (torch's fp64 matmul and log-softmax on the GPU): conf, ent,
+    tok and the top-2 gap.  Not the oracle: the caller pins it to the oracle on sampled rows."""
+    n = h_dev.shape[0]
+    wd = w_head.double()
+    conf = np.empty(n); ent = np.empty(n); tok = np.empty(n, np.int64); gap = np.empty(n)
+    for r0 in range(0, n, chunk):
+        lp = torch.log_softmax(h_dev[r0:r0 + chunk].double() @ wd.t(), dim=1)
+        top2 = lp.topk(2, dim=1)
+        conf[r0:r0 + chunk] = top2.values[:, 0].exp().cpu().numpy()
+        tok[r0:r0 + chunk] = top2.indices[:, 0].cpu().numpy()
+        gap[r0:r0 + chunk] = (top2.values[:, 0] - top2.values[:, 1]).cpu().numpy()
+        ent[r0:r0 + chunk] = (-(lp.exp() * lp).sum(dim=1)).cpu().numpy()
+        del lp
+    del wd
+    return conf, ent, tok, gap
+
+
+def test_config3_verification_pass_sampled():
+    # Config 3's verification pass at its stated size: the 64 sequences' (1 + K_t) * |R_b| rows (about 10^5, several
+    # passes over W of the 128-row kernel) scored in the geometry the benchmark times.  Sampled rows against the
+    # oracle one by one, every row against the torch fp64 reference that is pinned to the oracle on that sample, and
+    # pvf_verify on the GPU's own fp32 numbers against the oracle's rule fed the same numbers.
+    w_bits = synth.make_w(1001, synth.LLADA_VOCAB, synth.LLADA_HIDDEN)
+    st = synth.config3(w_bits=w_bits)
+    plan = st.plan_ids
+    p = st.params
+    K = int(p["budget"])
+    ctx = make_ctx(w_bits, plan, 131072, 64, 16)
+    prm = params_of(st)
+    seg, pos, act = t_i32(st.seg_off), t_i32(st.row_pos), t_u8(st.active)
+    sc = ctx.score(upload_bits(st.h_bits))
+    cm = ctx.commit(prm, seg, pos, act, sc["tok"], sc["conf"])
+    sel = ctx.select_drafts(prm, seg, pos, act, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
+    torch.cuda.synchronize()
+    g_sc, g_cm, gs = to_np(sc), to_np(cm), to_np(sel)
+    # the draft-pass decisions follow the oracle's rules on the GPU's own numbers (the scores themselves are checked
+    # in test_config3_large_batch_sampled)
+    ocm = ostep.commit(g_sc["conf"], g_sc["tok"], st.seg_off, st.row_pos, st.active, p["tau_high"])
+    osel = ostep.select_drafts(g_sc["conf"], g_sc["tok"], g_sc["in_plan"], ocm["commit"], st.seg_off, st.row_pos,
+                               st.active, p["tau_plan_lo"], p["tau_plan_hi"], p["tau_ar_lo"], K)
+    assert np.array_equal(g_cm["commit"], ocm["commit"])
+    for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+        assert np.array_equal(gs[k], osel[k]), k
+    n_rem = int(osel["rem_off"][-1])
+    assert np.array_equal(gs["rem_rows"][:n_rem], osel["rem_rows"][:n_rem])
+    v = synth.make_verify_pass(st, osel["rem_rows"], osel["rem_off"], osel["n_drafts"])
+    Mv = int(v.hv_bits.shape[0])
+    assert np.array_equal(v.v_off, osel["v_off"]) and Mv > 65536
+    geo = ctx.score_plan(Mv)
+    assert geo["waves"] >= 8 and ctx.score_kernel_name(Mv) == "pvf_score_gemm_kernel"
+    hv = upload_bits(v.hv_bits)
+    scv = ctx.score(hv)
+    ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"])
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    g_scv, gv = to_np(scv), to_np(ver)
+    check_score_properties(g_scv, st.vocab, plan)
+    # sampled rows: first and last row, both sides of a 128-row tile edge, of a wave edge (rows per pass over W) and
+    # of sequence boundaries of the [b][c][r] layout
+    rows_per_wave = 128 * ((Mv + 127) // 128 + geo["waves"] - 1) // geo["waves"]
+    rows_per_wave = min(rows_per_wave, Mv - 1)
+    sample = np.unique(np.clip(np.array([0, 127, 128, rows_per_wave - 1, rows_per_wave, int(v.v_off[1]) - 1, int(v.v_off[1]),
+                                         int(v.v_off[32]), Mv // 2, Mv - 129, Mv - 128, Mv - 1]), 0, Mv - 1))
+    want = oscore.score(w_bits, v.hv_bits[sample], plan)
+    check_score(g_scv, want, st.vocab, plan, rows=sample)
+    ref_conf, ref_ent, ref_tok, ref_gap = torch_fp64_reference(ctx.w_head, hv)
+    assert np.max(np.abs(ref_conf[sample] - want["conf"])) < 1e-9 and np.max(np.abs(ref_ent[sample] - want["ent"])) < 1e-9
+    assert np.array_equal(ref_tok[sample], want["tok"])
+    assert np.max(np.abs(g_scv["conf"] - ref_conf)) <= 1e-3 and np.max(np.abs(g_scv["ent"] - ref_ent)) <= 1e-3
+    clear = ref_gap >= NEAR_TIE
+    assert np.array_equal(g_scv["tok"][clear], ref_tok[clear]) and (~clear).sum() < 300
+    # acceptance, branch choice and final commit: the oracle's rule on the GPU's own verification-pass numbers
+    over = ostep.verify(g_sc["tok"], ocm["commit"], st.seg_off, st.row_pos, osel["rem_rows"], osel["rem_off"], osel["v_off"],
+                        osel["draft_rows"], osel["n_drafts"], osel["route"], g_scv["tok"], g_scv["conf"].astype(np.float64),
+                        p["tau_high"], K)
+    for k in ("accept", "choice", "final_commit"):
+        assert np.array_equal(gv[k], over[k]), k
+    assert (osel["route"] > 0).sum() >= st.n_seq // 2                  # the pass is not an empty formality
+    ctx.close()

@@ -9,8 +9,9 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import score as oscore
 from paper_2601_12247_b200 import binding, synth
-from gpu_util import TOL, dev, make_ctx, to_np, upload_bits
+from gpu_util import TOL, check_score, dev, make_ctx, to_np, upload_bits
 
 pytestmark = pytest.mark.gpu
 
@@ -88,3 +89,28 @@ def test_llada_shape_two_calls():
         assert binding.score_static_status() == 0
         compare(out, ctx.score(h))
     ctx.close()
+
+
+def test_matches_the_oracle_directly_and_allocates_no_device_memory():
+    # The property the entry point exists for: once a device has made its first call, further calls leave the
+    # amount of free device memory exactly as it was (cudaMemGetInfo through torch), whatever the row count and
+    # the kernel that serves it.  And its outputs are checked against the fp64 oracle itself, not only against
+    # pvf_score.
+    V, D, M_max = 4096, 256, 300
+    pos = np.arange(M_max)
+    st = synth.build_step("static-oracle", 778, V, D, 64, [(pos, np.ones(M_max, np.uint8))], M_max, M_max,
+                          dict(tau_high=0.9, budget=4))
+    w = upload_bits(st.w_bits)
+    bitmap = bitmap_of(st.plan_ids, V)
+    cases = [(M, upload_bits(st.h_bits[:M]), outputs(M)) for M in (150, 20, 300, 64)]   # every tensor exists beforehand
+    assert binding.score_static(w, cases[0][1], cases[0][2], bitmap) == binding.PVF_OK  # the device's set-up call
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for M, h, out in cases:
+        assert binding.score_static(w, h, out, bitmap) == binding.PVF_OK
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert binding.score_static_status() == 0
+    for M, h, out in cases:
+        check_score(to_np(out), oscore.score(st.w_bits, st.h_bits[:M], st.plan_ids), V, st.plan_ids)
