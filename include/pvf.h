@@ -16,7 +16,9 @@
  *   pvf_explore_commit     the appendix's Random / Planning exploration variants
  *   pvf_calib_accumulate, pvf_calib_filter, pvf_set_plan_bitmap
  *                          offline construction of the planning-token vocabulary
- *   pvf_draft_step_host, pvf_verify_step_host      the step with host buffers
+ *   pvf_commit_select      pvf_commit + pvf_select_drafts in one launch
+ *   pvf_draft_step, pvf_verify_step                the step as two calls of two launches each, device buffers
+ *   pvf_draft_step_host, pvf_verify_step_host      the same with host buffers
  *   pvf_score_static       scoring without a context, for callers that must not allocate
  *
  * Conventions common to all calls
@@ -114,14 +116,16 @@ int pvf_create(pvf_ctx **out, const pvf_shape *shape, const void *w_head,
                const int32_t *plan_ids_host, int32_t n_plan, void *workspace, size_t workspace_bytes);
 int pvf_destroy(pvf_ctx *ctx);
 
-/* Copies the device status word to *status (PVF_OK or PVF_ERR_TIMEOUT) and clears it.
- * Synchronises the device. */
+/* Copies the device status word to *status (PVF_OK or PVF_ERR_TIMEOUT) and clears it.  Synchronises the whole
+ * device first (cudaDeviceSynchronize: streams created non-blocking included).  Results of a call that timed
+ * out are undefined. */
 int pvf_last_status(pvf_ctx *ctx, int32_t *status);
 
 /*
  * Launch geometry pvf_score would use for M rows; any pointer may be NULL.
- *   ctas        thread blocks of the GEMM kernel            splits   vocabulary ranges per row tile
- *   waves       passes over the weight matrix               launches kernels launched per call
+ *   ctas        thread blocks of the projection kernel      splits   vocabulary ranges per row tile
+ *   waves       passes over the weight matrix               launches kernels launched per call (the projection
+ *                                                                    kernel and the merge of the ranges' states)
  */
 int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int32_t *waves, int32_t *launches);
 
@@ -200,6 +204,18 @@ int pvf_select_drafts(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t
                       int32_t *rem_rows, int32_t *rem_off, int32_t *v_off, void *stream);
 
 /*
+ * pvf_commit_select -- pvf_commit followed by pvf_select_drafts in ONE launch (Sections 2, 3, 4.1 and 4.3 as
+ * in those two calls; arguments, outputs and results are theirs, bit for bit).  One thread block per sequence
+ * takes the base set and then proposes the drafts from it.
+ */
+int pvf_commit_select(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
+                      const int32_t *seg_off, const int32_t *row_pos, const uint8_t *active,
+                      const int32_t *tok, const float *conf, const uint8_t *in_plan,
+                      uint8_t *commit, int32_t *n_commit, int32_t *y, int32_t L,
+                      int32_t *draft_rows, int32_t *n_drafts, uint8_t *route,
+                      int32_t *rem_rows, int32_t *rem_off, int32_t *v_off, void *stream);
+
+/*
  * pvf_verify -- acceptance check and final commit (Eq. 1 impact set, Eq. 3 verified compatibility,
  * Section 4.2 Filter 1 and Filter 2, Section 4.3 AR verification and selection).
  *   tok_v, conf_v   pvf_score outputs of the verification pass, rows [b][c][r]: index
@@ -222,6 +238,34 @@ int pvf_verify(pvf_ctx *ctx, const pvf_params *params, int32_t M, int32_t n_seq,
                const int32_t *tok, const int32_t *tok_v, const float *conf_v, const uint8_t *commit,
                uint8_t *accept, int32_t *choice, uint8_t *final_commit,
                int32_t *y, int32_t L, void *stream);
+
+/*
+ * One decoding iteration of Algorithm 1 as two calls around the model's verification forward, on device
+ * buffers, two kernel launches each: the projection kernel of pvf_score, and one kernel that first merges the
+ * projection's per-vocabulary-range softmax states (what pvf_score's own small second kernel does) and then
+ * takes the decisions -- results equal to the calls they combine, bit for bit.
+ *   pvf_draft_step    = pvf_score(hidden) + pvf_commit + pvf_select_drafts: scores of the draft pass (tok, conf,
+ *                     in_plan [M]; ent [M] or NULL), base set, drafts, and the row layout (rem_rows, rem_off,
+ *                     v_off) of the verification pass.  seg_off[n_seq] must equal M: every scored row belongs
+ *                     to a sequence (the rows are merged sequence by sequence).
+ *   pvf_verify_step   = pvf_score(hidden_v) + pvf_verify: scores of the verification rows (tok_v, conf_v [Mv];
+ *                     ent_v [Mv] or NULL), acceptance, branch choice, final commit.  Mv must equal the draft
+ *                     half's v_off[n_seq] (a device value the caller reads back to size the forward pass).
+ * Other arguments as in the calls they combine; asynchronous on `stream` like them.
+ */
+int pvf_draft_step(pvf_ctx *ctx, const pvf_params *params, const void *hidden, int32_t M, int32_t n_seq,
+                   const int32_t *seg_off, const int32_t *row_pos, const uint8_t *active,
+                   int32_t *tok, float *conf, float *ent, uint8_t *in_plan,
+                   uint8_t *commit, int32_t *n_commit, int32_t *y, int32_t L,
+                   int32_t *draft_rows, int32_t *n_drafts, uint8_t *route,
+                   int32_t *rem_rows, int32_t *rem_off, int32_t *v_off, void *stream);
+int pvf_verify_step(pvf_ctx *ctx, const pvf_params *params, const void *hidden_v, int32_t Mv, int32_t M, int32_t n_seq,
+                    const int32_t *seg_off, const int32_t *row_pos,
+                    const int32_t *rem_rows, const int32_t *rem_off, const int32_t *v_off,
+                    const int32_t *draft_rows, const int32_t *n_drafts, const uint8_t *route,
+                    const int32_t *tok, const uint8_t *commit,
+                    int32_t *tok_v, float *conf_v, float *ent_v,
+                    uint8_t *accept, int32_t *choice, uint8_t *final_commit, int32_t *y, int32_t L, void *stream);
 
 /*
  * pvf_explore_commit -- the exploration variants of the appendix ("Planning tokens beyond high-confidence
@@ -330,9 +374,9 @@ int pvf_working_set(pvf_ctx *ctx, const int32_t *y, int32_t n_seq, int32_t L, in
  *                            small input arrays travel as one host-to-device copy and all outputs of a call as
  *                            one device-to-host copy into the buffer, from which they are copied to the output
  *                            pointers (which then need not be pinned); without it every array is copied on its own.
- *   pvf_draft_step_host      pvf_score + pvf_commit + pvf_select_drafts on hidden_host[M][hidden]; outputs
- *                            as in those calls.  The device copies stay in the staging buffer.
- *   pvf_verify_step_host     pvf_score on hidden_v_host[Mv][hidden] + pvf_verify, continuing the draft
+ *   pvf_draft_step_host      pvf_draft_step on hidden_host[M][hidden]; outputs as there.  The device copies
+ *                            stay in the staging buffer.
+ *   pvf_verify_step_host     pvf_verify_step on hidden_v_host[Mv][hidden], continuing the draft
  *                            half most recently run on this context (same budget); Mv must equal that
  *                            half's v_off[n_seq].
  */
@@ -358,8 +402,8 @@ int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hid
  * loaded into a host process that forbids allocation after start-up, and latency-critical serving loops
  * where an allocation (and the implicit device synchronisation it can cause) is not acceptable.  pvf_score
  * asks such callers for a workspace through pvf_create; this entry point needs neither a context nor a
- * workspace.  Its scratch memory -- the per-vocabulary-range softmax states that the GEMM kernel writes and
- * the merge kernel reads -- is a fixed 512.25 KiB array inside the library image.  Every GPU that loads
+ * workspace.  Its scratch memory -- the per-vocabulary-range softmax states that the projection kernel writes
+ * and the merge kernel reads, and a status word -- is a fixed 512.25 KiB array inside the library image.  Every GPU that loads
  * the library holds that array until the process exits, whether or not this function is ever called.
  * (The array holds one state per row and SM.  Where pvf_score would pick the kernel that leaves two, and they
  * do not fit -- more than 221 rows -- this entry point takes the kernel pvf_score uses outside that window:
@@ -375,8 +419,9 @@ int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hid
  * The call itself allocates nothing: no cudaMalloc / cudaFree, no allocating library routine; it
  * encodes its tensor maps on the host, clears one status word with cudaMemsetAsync and launches the two
  * scoring kernels on `stream`.  The first call on each device additionally looks up the array's device
- * address and raises the GEMM kernel's shared-memory limit (this also makes the CUDA runtime load the
- * kernels); make that first call with the device current and before any stream capture begins.
+ * address and raises the scoring kernels' shared-memory limit (this also makes the CUDA runtime load the
+ * kernels); make that first call with the device current and before any stream capture begins.  That set-up
+ * is guarded by a lock, so several host threads may make their first calls at the same time.
  *
  * All calls on a device share the one array, and it keeps the last call's contents.  Only the status word
  * has to start from zero and the call clears it; the softmax states are fully rewritten before they are

@@ -86,6 +86,12 @@ def load() -> ctypes.CDLL:
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
         lib.pvf_verify.argtypes = [vp, pp, i32, i32] + [vp] * 16 + [i32, vp]; lib.pvf_verify.restype = ctypes.c_int
+        lib.pvf_commit_select.argtypes = [vp, pp, i32, i32] + [vp] * 9 + [i32] + [vp] * 6 + [vp]
+        lib.pvf_commit_select.restype = ctypes.c_int
+        lib.pvf_draft_step.argtypes = [vp, pp, vp, i32, i32] + [vp] * 10 + [i32] + [vp] * 6 + [vp]
+        lib.pvf_draft_step.restype = ctypes.c_int
+        lib.pvf_verify_step.argtypes = [vp, pp, vp, i32, i32, i32] + [vp] * 17 + [i32, vp]
+        lib.pvf_verify_step.restype = ctypes.c_int
         lib.pvf_explore_commit.argtypes = [vp, pp, i32, i32, i32] + [vp] * 10 + [i32, vp]
         lib.pvf_explore_commit.restype = ctypes.c_int
         pc = ctypes.POINTER(pvf_calib_params)
@@ -345,6 +351,73 @@ class Context:
                                         _ptr(out["draft_rows"]), _ptr(out["n_drafts"]), _ptr(out["route"]),
                                         _ptr(out["rem_rows"]), _ptr(out["rem_off"]), _ptr(out["v_off"]), _stream())
         _check(rc, "pvf_select_drafts")
+        return out
+
+    def _step_outputs(self, M: int, n_seq: int, K: int) -> Dict[str, torch.Tensor]:
+        dev = self.device
+        return dict(commit=torch.empty(M, dtype=torch.uint8, device=dev),
+                    n_commit=torch.empty(n_seq, dtype=torch.int32, device=dev),
+                    draft_rows=torch.empty((n_seq, K), dtype=torch.int32, device=dev),
+                    n_drafts=torch.empty(n_seq, dtype=torch.int32, device=dev),
+                    route=torch.empty(n_seq, dtype=torch.uint8, device=dev),
+                    rem_rows=torch.empty(max(M, 1), dtype=torch.int32, device=dev),
+                    rem_off=torch.empty(n_seq + 1, dtype=torch.int32, device=dev),
+                    v_off=torch.empty(n_seq + 1, dtype=torch.int32, device=dev))
+
+    def commit_select(self, params: pvf_params, seg_off, row_pos, active, tok, conf, in_plan, y=None, out=None):
+        """pvf_commit_select: pvf_commit + pvf_select_drafts in one launch; ``out`` holds both calls' outputs."""
+        M, n_seq, K = conf.shape[0], seg_off.shape[0] - 1, int(params.budget)
+        if out is None:
+            out = self._step_outputs(M, n_seq, K)
+        L = 0 if y is None else y.shape[1]
+        rc = self.lib.pvf_commit_select(self.handle, ctypes.byref(params), M, n_seq, _ptr(seg_off), _ptr(row_pos),
+                                        _ptr(active), _ptr(tok), _ptr(conf), _ptr(in_plan), _ptr(out["commit"]),
+                                        _ptr(out.get("n_commit")), _ptr(y), L, _ptr(out["draft_rows"]), _ptr(out["n_drafts"]),
+                                        _ptr(out["route"]), _ptr(out["rem_rows"]), _ptr(out["rem_off"]), _ptr(out["v_off"]),
+                                        _stream())
+        _check(rc, "pvf_commit_select")
+        return out
+
+    def draft_step(self, params: pvf_params, hidden, seg_off, row_pos, active, y=None, out=None):
+        """pvf_draft_step: pvf_score + pvf_commit_select (two launches).  ``out`` holds tok, conf, ent, in_plan and the
+        outputs of commit_select."""
+        M, n_seq, K = hidden.shape[0], seg_off.shape[0] - 1, int(params.budget)
+        if out is None:
+            out = self._step_outputs(M, n_seq, K)
+            out.update(tok=torch.empty(M, dtype=torch.int32, device=self.device),
+                       conf=torch.empty(M, dtype=torch.float32, device=self.device),
+                       ent=torch.empty(M, dtype=torch.float32, device=self.device),
+                       in_plan=torch.empty(M, dtype=torch.uint8, device=self.device))
+        L = 0 if y is None else y.shape[1]
+        rc = self.lib.pvf_draft_step(self.handle, ctypes.byref(params), _ptr(hidden), M, n_seq, _ptr(seg_off), _ptr(row_pos),
+                                     _ptr(active), _ptr(out["tok"]), _ptr(out["conf"]), _ptr(out.get("ent")), _ptr(out["in_plan"]),
+                                     _ptr(out["commit"]), _ptr(out.get("n_commit")), _ptr(y), L, _ptr(out["draft_rows"]),
+                                     _ptr(out["n_drafts"]), _ptr(out["route"]), _ptr(out["rem_rows"]), _ptr(out["rem_off"]),
+                                     _ptr(out["v_off"]), _stream())
+        _check(rc, "pvf_draft_step")
+        return out
+
+    def verify_step(self, params: pvf_params, hidden_v, seg_off, row_pos, draft: Dict[str, torch.Tensor], y=None, out=None):
+        """pvf_verify_step: pvf_score on the verification pass + pvf_verify (two launches).  ``draft`` is the
+        output of draft_step (or of score + commit_select); ``out`` holds tok_v, conf_v, accept, choice, final_commit."""
+        Mv = 0 if hidden_v is None else hidden_v.shape[0]
+        M, n_seq, K = draft["commit"].shape[0], seg_off.shape[0] - 1, int(params.budget)
+        if out is None:
+            dev = self.device
+            out = dict(tok_v=torch.empty(max(Mv, 1), dtype=torch.int32, device=dev),
+                       conf_v=torch.empty(max(Mv, 1), dtype=torch.float32, device=dev),
+                       ent_v=torch.empty(max(Mv, 1), dtype=torch.float32, device=dev),
+                       accept=torch.empty((n_seq, K), dtype=torch.uint8, device=dev),
+                       choice=torch.empty(n_seq, dtype=torch.int32, device=dev),
+                       final_commit=torch.empty(M, dtype=torch.uint8, device=dev))
+        L = 0 if y is None else y.shape[1]
+        rc = self.lib.pvf_verify_step(self.handle, ctypes.byref(params), _ptr(hidden_v), Mv, M, n_seq, _ptr(seg_off),
+                                      _ptr(row_pos), _ptr(draft["rem_rows"]), _ptr(draft["rem_off"]), _ptr(draft["v_off"]),
+                                      _ptr(draft["draft_rows"]), _ptr(draft["n_drafts"]), _ptr(draft["route"]),
+                                      _ptr(draft["tok"]), _ptr(draft["commit"]), _ptr(out["tok_v"]), _ptr(out["conf_v"]),
+                                      _ptr(out.get("ent_v")), _ptr(out["accept"]), _ptr(out["choice"]), _ptr(out["final_commit"]),
+                                      _ptr(y), L, _stream())
+        _check(rc, "pvf_verify_step")
         return out
 
     def verify(self, params: pvf_params, seg_off, row_pos, sel: Dict[str, torch.Tensor], tok, tok_v, conf_v,

@@ -7,8 +7,8 @@
 namespace {
 
 struct Layout {
-    size_t words_off, bitmap_off, partials_off, total;
-    size_t bitmap_bytes, partials_bytes;
+    size_t words_off, bitmap_off, seq_tickets_off, partials_off, total;
+    size_t bitmap_bytes, seq_tickets_bytes, partials_bytes;
 };
 
 bool shape_ok(const pvf_shape *s)
@@ -23,7 +23,9 @@ Layout layout_for(const pvf_shape *s, int n_sm)
     l.words_off = 0;
     l.bitmap_off = pvf_align_up(sizeof(pvf_device_words), 256);
     l.bitmap_bytes = pvf_align_up(((size_t)s->vocab + 31) / 32 * 4, 256);
-    l.partials_off = l.bitmap_off + l.bitmap_bytes;
+    l.seq_tickets_off = l.bitmap_off + l.bitmap_bytes;
+    l.seq_tickets_bytes = pvf_align_up(((size_t)s->max_seqs + 1) * sizeof(uint32_t), 256);
+    l.partials_off = l.seq_tickets_off + l.seq_tickets_bytes;
     l.partials_bytes = pvf_align_up(pvf_score_partials_bytes(s, n_sm), 256);
     l.total = l.partials_off + l.partials_bytes;
     return l;
@@ -102,6 +104,8 @@ int pvf_create(pvf_ctx **out, const pvf_shape *shape, const void *w_head,
     ctx->workspace_bytes = workspace_bytes;
     ctx->words = (pvf_device_words *)(ctx->workspace + l.words_off);
     ctx->plan_bitmap = (uint32_t *)(ctx->workspace + l.bitmap_off);
+    ctx->seq_tickets = (uint32_t *)(ctx->workspace + l.seq_tickets_off);
+    ctx->seq_tickets_bytes = l.seq_tickets_bytes;
     ctx->partials = (float4 *)(ctx->workspace + l.partials_off);
     ctx->partials_bytes = l.partials_bytes;
     ctx->ev_start = nullptr;
@@ -115,6 +119,7 @@ int pvf_create(pvf_ctx **out, const pvf_shape *shape, const void *w_head,
     std::vector<uint32_t> bitmap(l.bitmap_bytes / 4, 0u);
     for (int32_t i = 0; i < n_plan; ++i) bitmap[plan_ids_host[i] >> 5] |= 1u << (plan_ids_host[i] & 31);
     bool ok = cudaMemset(ctx->words, 0, sizeof(pvf_device_words)) == cudaSuccess &&
+              cudaMemset(ctx->seq_tickets, 0, l.seq_tickets_bytes) == cudaSuccess &&
               cudaMemcpy(ctx->plan_bitmap, bitmap.data(), l.bitmap_bytes, cudaMemcpyHostToDevice) == cudaSuccess &&
               cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) { delete ctx; return PVF_ERR_CUDA; }
@@ -134,8 +139,17 @@ int pvf_last_status(pvf_ctx *ctx, int32_t *status)
 {
     if (!ctx || !status) return PVF_ERR_INVALID;
     int32_t host = 0;
+    // Every stream of the device, non-blocking ones included: a copy on the legacy default stream alone would
+    // not wait for kernels launched on those.
+    if (cudaDeviceSynchronize() != cudaSuccess) return PVF_ERR_CUDA;
     if (cudaMemcpy(&host, &ctx->words->status, sizeof host, cudaMemcpyDeviceToHost) != cudaSuccess) return PVF_ERR_CUDA;
-    if (host != 0 && cudaMemset(&ctx->words->status, 0, sizeof(int32_t)) != cudaSuccess) return PVF_ERR_CUDA;
+    if (host != 0) {
+        // A kernel gave up: clear the word (and the arrival tickets, which count whole blocks and so stay whole).
+        if (cudaMemset(&ctx->words->status, 0, sizeof(int32_t)) != cudaSuccess ||
+            cudaMemset(&ctx->words->select_ticket, 0, 2 * sizeof(uint32_t)) != cudaSuccess ||
+            cudaMemset(ctx->seq_tickets, 0, ctx->seq_tickets_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
+            return PVF_ERR_CUDA;
+    }
     *status = host;
     return PVF_OK;
 }

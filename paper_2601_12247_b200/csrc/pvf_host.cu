@@ -1,7 +1,7 @@
-// Host-buffer variants of the step: inputs and outputs live in host memory, the library stages them
-// through a caller-provided device buffer with cudaMemcpyAsync and synchronises the stream before
-// returning.  The arithmetic is the device entry points' (pvf_score, pvf_commit, pvf_select_drafts,
-// pvf_verify); nothing is computed on the host.
+// Host-buffer variants of the step calls (pvf_draft_step, pvf_verify_step): inputs and outputs live in host
+// memory, the library stages them through a caller-provided device buffer with cudaMemcpyAsync and
+// synchronises the stream before returning.  The arithmetic is the device entry points'; nothing is
+// computed on the host.
 #include <string.h>
 
 #include "pvf_internal.h"
@@ -137,17 +137,11 @@ int pvf_draft_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hidd
                !h2d(g + l.row_pos, row_pos_host, (size_t)M * 4, s) ||
                (active_host && !h2d(g + l.active, active_host, (size_t)M, s)))
         return PVF_ERR_CUDA;
-    int rc = pvf_score(ctx, g + l.hidden, M, (int32_t *)(g + l.tok), (float *)(g + l.conf), (float *)(g + l.ent),
-                       g + l.in_plan, stream);
-    if (rc != PVF_OK) return rc;
-    rc = pvf_commit(ctx, params, M, n_seq, (const int32_t *)(g + l.seg_off), (const int32_t *)(g + l.row_pos), active_dev,
-                    (const int32_t *)(g + l.tok), (const float *)(g + l.conf), g + l.commit, (int32_t *)(g + l.n_commit),
-                    nullptr, 0, stream);
-    if (rc != PVF_OK) return rc;
-    rc = pvf_select_drafts(ctx, params, M, n_seq, (const int32_t *)(g + l.seg_off), (const int32_t *)(g + l.row_pos),
-                           active_dev, (const int32_t *)(g + l.tok), (const float *)(g + l.conf), g + l.in_plan,
-                           g + l.commit, (int32_t *)(g + l.draft_rows), (int32_t *)(g + l.n_drafts), g + l.route,
-                           (int32_t *)(g + l.rem_rows), (int32_t *)(g + l.rem_off), (int32_t *)(g + l.v_off), stream);
+    int rc = pvf_draft_step(ctx, params, g + l.hidden, M, n_seq, (const int32_t *)(g + l.seg_off), (const int32_t *)(g + l.row_pos),
+                            active_dev, (int32_t *)(g + l.tok), (float *)(g + l.conf), (float *)(g + l.ent), g + l.in_plan,
+                            g + l.commit, (int32_t *)(g + l.n_commit), nullptr, 0, (int32_t *)(g + l.draft_rows),
+                            (int32_t *)(g + l.n_drafts), g + l.route, (int32_t *)(g + l.rem_rows), (int32_t *)(g + l.rem_off),
+                            (int32_t *)(g + l.v_off), stream);
     if (rc != PVF_OK) return rc;
     if (hb) {
         if (!d2h(hb + l.tok, g + l.tok, l.draft_end - l.tok, s) || cudaStreamSynchronize(s) != cudaSuccess) return PVF_ERR_CUDA;
@@ -195,13 +189,12 @@ int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hid
     cudaStream_t s = (cudaStream_t)stream;
     const size_t K = (size_t)params->budget;
     if (!h2d(g + l.hidden, hidden_v_host, (size_t)Mv * ctx->shape.hidden * 2, s)) return PVF_ERR_CUDA;
-    int rc = pvf_score(ctx, g + l.hidden, Mv, (int32_t *)(g + l.tok_v), (float *)(g + l.conf_v), nullptr, nullptr, stream);
-    if (rc != PVF_OK) return rc;
-    rc = pvf_verify(ctx, params, M, n_seq, (const int32_t *)(g + l.seg_off), (const int32_t *)(g + l.row_pos),
-                    (const int32_t *)(g + l.rem_rows), (const int32_t *)(g + l.rem_off), (const int32_t *)(g + l.v_off),
-                    (const int32_t *)(g + l.draft_rows), (const int32_t *)(g + l.n_drafts), g + l.route,
-                    (const int32_t *)(g + l.tok), (const int32_t *)(g + l.tok_v), (const float *)(g + l.conf_v), g + l.commit,
-                    g + l.accept, (int32_t *)(g + l.choice), g + l.final_commit, nullptr, 0, stream);
+    int rc = pvf_verify_step(ctx, params, g + l.hidden, Mv, M, n_seq, (const int32_t *)(g + l.seg_off),
+                             (const int32_t *)(g + l.row_pos), (const int32_t *)(g + l.rem_rows), (const int32_t *)(g + l.rem_off),
+                             (const int32_t *)(g + l.v_off), (const int32_t *)(g + l.draft_rows), (const int32_t *)(g + l.n_drafts),
+                             g + l.route, (const int32_t *)(g + l.tok), g + l.commit, (int32_t *)(g + l.tok_v),
+                             (float *)(g + l.conf_v), nullptr, g + l.accept, (int32_t *)(g + l.choice), g + l.final_commit,
+                             nullptr, 0, stream);
     if (rc != PVF_OK) return rc;
     if (hb) {
         if (!d2h(hb + l.accept, g + l.accept, l.total - l.accept, s) || cudaStreamSynchronize(s) != cudaSuccess) return PVF_ERR_CUDA;

@@ -28,6 +28,8 @@ struct pvf_ctx {
     size_t workspace_bytes;
     pvf_device_words *words;
     uint32_t *plan_bitmap;  // ceil(V/32) words, bit v set iff v in P^plan
+    uint32_t *seq_tickets;  // one arrival counter per sequence (step kernels; zero between launches)
+    size_t seq_tickets_bytes;
     float4 *partials;       // [rows][splits] per-range softmax states of pvf_score
     size_t partials_bytes;
     CUtensorMap tm_w[PVF_W_BOX_SIZES];   // W as [V][D], boxes of 16 * (i + 1) rows x 64 columns, 128-byte swizzle
@@ -61,6 +63,9 @@ struct pvf_score_geometry {
 pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool allow_swapped = true);
 size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm);
 int pvf_score_init(pvf_ctx *ctx);   // tensor maps of W, kernel attributes
+// The projection half of pvf_score alone: launches the kernel that leaves `*parts` partial softmax states per row in
+// ctx->partials (row stride *parts); the caller's next kernel on the stream merges them (pvf_merge_rows).
+int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, void *stream);
 
 // Programmatic dependent launch.  Every kernel of the library is launched with pvf_launch and runs
 //     <set-up that touches no global memory>; pvf_launch_dependents(); pvf_grid_dependency_wait();
@@ -108,6 +113,113 @@ static inline cudaError_t pvf_launch_cluster2(void (*kernel)(KArgs...), dim3 gri
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
+// Partial softmax state of a row over a vocabulary range, as the projection kernels leave it (one float4):
+//   x = the range's maximum logit m        y = sum of e^{x_v - m} over the range EXCEPT the entry holding the maximum
+//   z = sum of (x_v - m) e^{x_v - m}       w = bits of the lowest token id attaining m (kPvfNoArg: empty state)
+// Keeping the maximum's own term (1.0) out of y keeps the small terms of a peaked row above the rounding unit.
+#ifdef __CUDACC__
+constexpr int kPvfNoArg = 0x7fffffff;
+
+__device__ __forceinline__ float pvf_fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// a <- a merged with b (two states over disjoint vocabulary sets).  The larger max stays outside the sum; the
+// other state's max joins it as an ordinary term.  Equal maxima: the lower token id wins.  Branch-free, so that
+// independent merges interleave: the loser's distance below the winner is clamped (an empty state sits at -inf and
+// comes in with weight e^-inf = 0; two empty states give an empty state).
+__device__ __forceinline__ void pvf_state_merge(float4 &a, const float4 b)
+{
+    constexpr float kLog2e = 1.4426950408889634f;
+    const int ia = __float_as_int(a.w), ib = __float_as_int(b.w);
+    const bool a_wins = a.x > b.x || (a.x == b.x && ia <= ib);
+    const float wm = a_wins ? a.x : b.x, wy = a_wins ? a.y : b.y, wz = a_wins ? a.z : b.z, ww = a_wins ? a.w : b.w;
+    const float lm = a_wins ? b.x : a.x, ly = a_wins ? b.y : a.y, lz = a_wins ? b.z : a.z;
+    const float d = fmaxf(lm - wm, -1.0e30f);           // <= 0; fmaxf also turns (-inf) - (-inf) into the clamp
+    const float c = pvf_fast_exp2(d * kLog2e);
+    const float total = ly + 1.f;
+    a.x = wm;
+    a.y = fmaf(total, c, wy);
+    a.z = fmaf(fmaf(d, total, lz), c, wz);
+    a.w = ww;
+}
+
+// Final merge of rows [row_begin, row_end) by the warps of a block, or of a grid of such blocks (all threads call it;
+// `warp` / `n_warps` = this warp's index among the warps that share the row range).  A row's `parts` partial states
+// are folded by g = min(32, parts rounded up to a power of two) neighbouring lanes -- lane l takes states l, l + g,
+// ... in turn, then the lanes fold pairwise: an order fixed by `parts` alone, so results are identical from run to
+// run -- and the row's first lane writes token, confidence = 1 / (1 + y), entropy = ln(1 + y) - z / (1 + y) and
+// planning-vocabulary membership (Section 3: y^, p, H; Section 4.1: y^ in P^plan).  ent and in_plan may be NULL.
+// A warp works on kMergeRowsInFlight groups of 32 / g rows at once and fetches up to kMergeStatesInFlight states per
+// lane and row before it merges any (the merge is a chain of memory round trips otherwise).  No shared memory and
+// few registers: the kernels that run this are launched while the projection kernel, which fills an SM's shared
+// memory and two thirds of its registers, is still running, and their blocks must fit beside its blocks to be
+// resident (and past their set-up) by the time it ends.
+constexpr int kMergeRowsInFlight = 2;
+constexpr int kMergeStatesInFlight = 5;
+__device__ __forceinline__ void pvf_merge_rows(const float4 *__restrict__ partials, int parts, int vocab,
+                                               const uint32_t *__restrict__ plan_bitmap, int row_begin, int row_end,
+                                               int warp, int n_warps, int32_t *tok, float *conf, float *ent, uint8_t *in_plan)
+{
+    int g = 1;
+    while (g < parts && g < 32) g <<= 1;
+    const int lane = threadIdx.x & 31;
+    const int gl = lane & (g - 1), sub = lane / g;              // lane within its row, row within the warp's pass
+    const int rows_per_pass = 32 / g;
+    const int rows_per_turn = rows_per_pass * kMergeRowsInFlight;
+    const float4 none = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(kPvfNoArg));
+#pragma unroll 1
+    for (int row0 = row_begin + warp * rows_per_turn; row0 < row_end; row0 += n_warps * rows_per_turn) {
+        float4 acc[kMergeRowsInFlight];
+#pragma unroll
+        for (int r = 0; r < kMergeRowsInFlight; ++r) acc[r] = none;
+#pragma unroll 1
+        for (int i0 = gl; i0 < parts; i0 += g * kMergeStatesInFlight) {
+            float4 v[kMergeRowsInFlight][kMergeStatesInFlight];
+#pragma unroll
+            for (int r = 0; r < kMergeRowsInFlight; ++r) {
+                const int row = row0 + r * rows_per_pass + sub;
+#pragma unroll
+                for (int k = 0; k < kMergeStatesInFlight; ++k)
+                    v[r][k] = (row < row_end && i0 + k * g < parts) ? __ldg(partials + (size_t)row * parts + i0 + k * g) : none;
+            }
+#pragma unroll
+            for (int r = 0; r < kMergeRowsInFlight; ++r)
+#pragma unroll
+                for (int k = 0; k < kMergeStatesInFlight; ++k) pvf_state_merge(acc[r], v[r][k]);
+        }
+#pragma unroll
+        for (int r = 0; r < kMergeRowsInFlight; ++r) {
+#pragma unroll 1
+            for (int o = 1; o < g; o <<= 1) {                   // lane l absorbs lane l + o of its row
+                float4 other;
+                other.x = __shfl_down_sync(0xffffffffu, acc[r].x, o, g);
+                other.y = __shfl_down_sync(0xffffffffu, acc[r].y, o, g);
+                other.z = __shfl_down_sync(0xffffffffu, acc[r].z, o, g);
+                other.w = __shfl_down_sync(0xffffffffu, acc[r].w, o, g);
+                if ((gl & (2 * o - 1)) == 0) pvf_state_merge(acc[r], other);
+            }
+            const int row = row0 + r * rows_per_pass + sub;
+            if (gl == 0 && row < row_end) {
+                // A row of non-finite logits never sets a maximum: its outputs are unspecified, but the token stays a
+                // valid id and the bitmap lookup in bounds.
+                int arg = __float_as_int(acc[r].w);
+                if ((unsigned)arg >= (unsigned)vocab) arg = 0;
+                const float norm = 1.f + acc[r].y;              // the maximum's own term is the 1
+                const float inv = 1.f / norm;
+                tok[row] = arg;
+                conf[row] = inv;
+                if (ent) ent[row] = __logf(norm) - acc[r].z * inv;
+                if (in_plan) in_plan[row] = (uint8_t)((plan_bitmap[arg >> 5] >> (arg & 31)) & 1u);
+            }
+        }
+    }
 }
 #endif
 

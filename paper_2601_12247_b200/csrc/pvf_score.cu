@@ -7,7 +7,10 @@
 // vocabulary on its columns, so one epilogue thread owns one row and keeps that row's running
 // softmax state (max, argmax, sum e^{x-max}, sum (x-max) e^{x-max}) in registers while the thread
 // block sweeps a contiguous vocabulary range.  Each (row, range) pair leaves one 16-byte partial
-// state; a small second kernel merges the partials of a row.
+// state; the kernel that follows on the stream merges the partial states of a row: the small merge
+// kernel of pvf_score, or the head of the step kernels (pvf_draft_step: merge + commit + select in one
+// launch; pvf_verify_step: merge + verify), which then write token, confidence, entropy and planning-
+// vocabulary membership themselves.
 //
 // Thread block = 6 warps:  warp 0 issues TMA loads (W and H tiles, 128-byte swizzle, a ring of
 // stages), warp 1 owns tensor memory and issues the MMAs, warps 2-5 are the softmax epilogue.  Two
@@ -32,7 +35,12 @@
 // the status word, raises a block-wide abort flag, drains its outstanding copies and MMAs with
 // bounded waits, frees its tensor memory and returns.
 // The kernels live in pvf_score_*.cuh (one file each, all part of this translation unit); this file holds the
-// merge kernel, the host-side work split and the entry points.
+// merge kernel, the host-side work split and the entry points.  (Merging in the projection kernel's own tail, by the
+// block that finishes last, was built and measured: that code runs once per launch on instructions the weight
+// stream has long pushed out of L2, and cost 9 .. 30 us per call against 4 us for a kernel whose blocks are resident
+// and waiting -- programmatic dependent launch -- before the projection ends.)
+#include <mutex>
+
 #include "pvf_score_common.cuh"
 #include "pvf_score_gemm.cuh"
 #include "pvf_score_gemm_pair.cuh"
@@ -42,57 +50,18 @@
 namespace {
 
 // ---------------------------------------------------------------------------------- merge kernel
-// One warp per row: combines the row's `splits` partial states (any order: ties go to the lowest id) in
-// fp64 and writes token, confidence, entropy and planning-vocabulary membership.
-__global__ void __launch_bounds__(256)
-pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int splits, int vocab,
+// Combines the rows' partial states and writes token, confidence, entropy and planning-vocabulary membership.
+constexpr int kMergeKernelThreads = 128;
+__global__ void __launch_bounds__(kMergeKernelThreads, 1)
+pvf_score_merge_kernel(const float4 *__restrict__ partials, int M, int parts, int vocab,
                        const uint32_t *__restrict__ plan_bitmap, int32_t *__restrict__ tok,
                        float *__restrict__ conf, float *__restrict__ ent, uint8_t *__restrict__ in_plan)
 {
     pvf_launch_dependents();
     pvf_grid_dependency_wait();
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= M) return;
-    const float4 *p = partials + (size_t)row * splits;
-    // lane-local pass: only the max and its lowest id
-    float m = -INFINITY;
-    int arg = kNoArg;
-    for (int i = lane; i < splits; i += 32) {
-        const float4 v = p[i];
-        const int a = __float_as_int(v.w);
-        if (a != kNoArg && (v.x > m || (v.x == m && a < arg))) { m = v.x; arg = a; }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, m, o);
-        const int a2 = __shfl_xor_sync(0xffffffffu, arg, o);
-        if (m2 > m || (m2 == m && a2 < arg)) { m = m2; arg = a2; }
-    }
-    // rescale every partial to the global max and add; a partial's sum leaves out its own max's term (1)
-    double s = 0.0, t = 0.0;
-    for (int i = lane; i < splits; i += 32) {
-        const float4 v = p[i];
-        if (__float_as_int(v.w) != kNoArg) {
-            const double d = (double)v.x - (double)m;
-            const double c = exp(d);
-            const double total = 1.0 + (double)v.y;
-            s += total * c;
-            t += ((double)v.z + d * total) * c;
-        }
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-        s += __shfl_xor_sync(0xffffffffu, s, o);
-        t += __shfl_xor_sync(0xffffffffu, t, o);
-    }
-    if (lane == 0) {
-        // A row of non-finite logits never sets a maximum: its outputs are unspecified, but the token stays a
-        // valid id and the bitmap lookup in bounds.
-        if ((unsigned)arg >= (unsigned)vocab) arg = 0;
-        tok[row] = arg;
-        conf[row] = (float)(1.0 / s);
-        if (ent) ent[row] = (float)(log(s) - t / s);
-        if (in_plan) in_plan[row] = (uint8_t)((plan_bitmap[arg >> 5] >> (arg & 31)) & 1u);
-    }
+    const int warps_per_block = kMergeKernelThreads / 32;
+    pvf_merge_rows(partials, parts, vocab, plan_bitmap, 0, M, (int)blockIdx.x * warps_per_block + (int)(threadIdx.x >> 5),
+                   (int)gridDim.x * warps_per_block, tok, conf, ent, in_plan);
 }
 
 // ---------------------------------------------------------------------------------- host side
@@ -153,10 +122,9 @@ int raise_shared_memory_limits()
     return PVF_OK;
 }
 
-// Launches the GEMM kernel (shape chosen by the geometry) and the merge kernel on `s`.
-int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, int D, const CUtensorMap *w_levels,
-                 float4 *partials, int32_t *status, const uint32_t *plan_bitmap, int32_t *tok, float *conf, float *ent,
-                 uint8_t *in_plan, cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop)
+// Launches the projection kernel (shape chosen by the geometry) on `s`: it leaves g.parts partial states per row.
+int launch_projection(const pvf_score_geometry &g, const void *hidden, int M, int V, int D, const CUtensorMap *w_levels,
+                      float4 *partials, int32_t *status, cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop)
 {
     CUtensorMap tm_h;
     int rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)g.a_rows);
@@ -171,6 +139,7 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
     a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
     a.a_rows = g.a_rows;
     a.n_pad = g.n_pad; a.stages = g.stages; a.parts = g.parts;
+    a.w_once = (g.waves == 1 && g.mb == 1) ? 1 : 0;
     a.partials = partials;
     a.status = status;
     const bool timed = ev_start && ev_stop;
@@ -191,9 +160,22 @@ int launch_score(const pvf_score_geometry &g, const void *hidden, int M, int V, 
         e = pvf_launch(pvf_score_gemm_kernel<GeneralCfg>, dim3(g.ctas), dim3(kThreads), GeneralCfg::kSmemBytes, s, tm_h, maps, a);
     if (e != cudaSuccess) return PVF_ERR_CUDA;
     if (timed && cudaEventRecord(ev_stop, s) != cudaSuccess) return PVF_ERR_CUDA;
-    const int warps_per_block = 8;
-    e = pvf_launch(pvf_score_merge_kernel, dim3((M + warps_per_block - 1) / warps_per_block), dim3(warps_per_block * 32), 0, s,
-                   (const float4 *)partials, M, g.parts, V, plan_bitmap, tok, conf, ent, in_plan);
+    return PVF_OK;
+}
+
+// The merge kernel of pvf_score on `s`.
+int launch_merge(const float4 *partials, int M, int parts, int V, const uint32_t *plan_bitmap, int32_t *tok, float *conf,
+                 float *ent, uint8_t *in_plan, cudaStream_t s)
+{
+    // one turn of a warp covers kMergeRowsInFlight groups of 32 / g rows (g lanes per row)
+    int g = 1;
+    while (g < parts && g < 32) g <<= 1;
+    const int rows_per_turn = (32 / g) * kMergeRowsInFlight, warps_per_block = kMergeKernelThreads / 32;
+    const int turns = (M + rows_per_turn - 1) / rows_per_turn;
+    int blocks = (turns + warps_per_block - 1) / warps_per_block;
+    blocks = blocks > 1184 ? 1184 : blocks;                            // the warps stride over the rows beyond that
+    const cudaError_t e = pvf_launch(pvf_score_merge_kernel, dim3(blocks), dim3(kMergeKernelThreads), 0, s, partials, M, parts, V,
+                                     plan_bitmap, tok, conf, ent, in_plan);
     return e == cudaSuccess ? PVF_OK : PVF_ERR_CUDA;
 }
 
@@ -245,7 +227,7 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool al
     g.a_rows = tiles128 == 1 ? ((M + 7) / 8) * 8 : kTileM;
     SplitPlan p = plan_split(M, V, D, n_sm, kTileM, kUnit, kMaxConcurrentTiles);
     g.paired = 0;
-    if (tiles128 >= PVF_PAIR_MIN_TILES && M <= PVF_PAIR_MAX_ROWS && n_sm >= 2) {
+    if (tiles128 >= kPairMinTiles && M <= kPairMaxRows && n_sm >= 2) {
         // The paired kernel works on 256-row tiles, granules of 32 vocabulary entries and pairs of SMs.  It
         // feeds the tensor cores better (measured: +8 .. +29 % from 129 to 8192 rows); it loses where pairs
         // and 256-row tiles divide the work less evenly, and in long launches the power cap, not the operand
@@ -254,8 +236,8 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool al
         if (pp.waves > 0 && pp.cost <= 1.05 * p.cost) { p = pp; g.paired = 1; }
     }
     g.swapped = 0; g.n_pad = 0; g.stages = 0;
-    if (allow_swapped && n_sm >= 2 && ((M > kStreamRows && M <= PVF_SWAP_SMALL_MAX_ROWS) || (M > kTileM && M <= PVF_SWAP_RAGGED_MAX_ROWS) ||
-                      (M > kSwapGroupCols && M <= PVF_SWAP_WIDE_MAX_ROWS))) {
+    if (allow_swapped && n_sm >= 2 && ((M > kStreamRows && M <= kSwapSmallMaxRows) || (M > kTileM && M <= kSwapRaggedMaxRows) ||
+                      (M > kSwapGroupCols && M <= kSwapWideMaxRows))) {
         // Swapped paired kernel: all rows, padded to a multiple of 32, are accumulator columns; every pair of SMs
         // sweeps one vocabulary range.  Chosen where the other kernels pad the rows most or sweep W twice (see the kernel).
         g.swapped = 1; g.paired = 0;
@@ -281,9 +263,9 @@ size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm)
     // every 128-row step and of the swapped paired kernel's two windows.
     for (int t = 1; t <= max_tiles + 3; ++t) {
         int rows = t * kTileM;
-        if (t == max_tiles + 1) rows = PVF_SWAP_SMALL_MAX_ROWS;
-        if (t == max_tiles + 2) rows = PVF_SWAP_RAGGED_MAX_ROWS;
-        if (t == max_tiles + 3) rows = PVF_SWAP_WIDE_MAX_ROWS;
+        if (t == max_tiles + 1) rows = kSwapSmallMaxRows;
+        if (t == max_tiles + 2) rows = kSwapRaggedMaxRows;
+        if (t == max_tiles + 3) rows = kSwapWideMaxRows;
         if (rows > shape->max_rows) rows = shape->max_rows;
         if (rows <= 0) continue;
         const pvf_score_geometry g = pvf_score_geometry_for(rows, shape->vocab, shape->hidden, n_sm);
@@ -291,6 +273,18 @@ size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm)
         worst = need > worst ? need : worst;
     }
     return worst;
+}
+
+int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, void *stream)
+{
+    if (!ctx || !parts || M <= 0 || M > ctx->shape.max_rows || !hidden) return PVF_ERR_INVALID;
+    if (((uintptr_t)hidden & 15) != 0) return PVF_ERR_ALIGN;
+    const int V = ctx->shape.vocab, D = ctx->shape.hidden;
+    const pvf_score_geometry g = pvf_score_geometry_for(M, V, D, ctx->n_sm);
+    if ((size_t)M * g.parts * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
+    *parts = g.parts;
+    return launch_projection(g, hidden, M, V, D, ctx->tm_w, ctx->partials, &ctx->words->status, (cudaStream_t)stream,
+                             ctx->ev_start, ctx->ev_stop);
 }
 
 int pvf_score_init(pvf_ctx *ctx)
@@ -349,12 +343,10 @@ int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
     if (!ctx || M < 0 || M > ctx->shape.max_rows) return PVF_ERR_INVALID;
     if (M == 0) return PVF_OK;
     if (!hidden || !tok || !conf) return PVF_ERR_INVALID;
-    if (((uintptr_t)hidden & 15) != 0) return PVF_ERR_ALIGN;
-    const int V = ctx->shape.vocab, D = ctx->shape.hidden;
-    const pvf_score_geometry g = pvf_score_geometry_for(M, V, D, ctx->n_sm);
-    if ((size_t)M * g.parts * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
-    return launch_score(g, hidden, M, V, D, ctx->tm_w, ctx->partials, &ctx->words->status, ctx->plan_bitmap, tok, conf,
-                        ent, in_plan, (cudaStream_t)stream, ctx->ev_start, ctx->ev_stop);
+    int parts = 0;
+    const int rc = pvf_score_partials(ctx, hidden, M, &parts, stream);
+    if (rc != PVF_OK) return rc;
+    return launch_merge(ctx->partials, M, parts, ctx->shape.vocab, ctx->plan_bitmap, tok, conf, ent, in_plan, (cudaStream_t)stream);
 }
 
 }  // extern "C"
@@ -370,7 +362,8 @@ constexpr size_t kStaticHeaderBytes = 256;                      // status word, 
 constexpr size_t kStaticPartialsBytes = (size_t)kTileM * kStaticMaxSms * sizeof(float4);
 constexpr int kStaticMaxDevices = 64;
 
-// Every GPU that loads this library holds these 512.25 KiB until the process exits.
+// Every GPU that loads this library holds these 512.25 KiB until the process exits: a 256-byte header (the status
+// word), then 128 x 256 partial softmax states.
 static __device__ __align__(256) unsigned char pvf_static_scratch[kStaticHeaderBytes + kStaticPartialsBytes];
 
 struct StaticDeviceState {
@@ -379,6 +372,7 @@ struct StaticDeviceState {
     unsigned char *scratch;     // device address of pvf_static_scratch on that GPU
 };
 StaticDeviceState g_static_state[kStaticMaxDevices];
+std::mutex g_static_mutex;          // guards the set-up below: first calls may come from several host threads
 
 // Once per device, with that device current: resolve the array's device address (its name is only a
 // host-side handle here) and raise the GEMM kernels' shared-memory limit.
@@ -388,6 +382,7 @@ int static_device_state(StaticDeviceState **out)
     if (cudaGetDevice(&device) != cudaSuccess) return PVF_ERR_CUDA;
     if (device < 0 || device >= kStaticMaxDevices) return PVF_ERR_UNSUPPORTED;
     StaticDeviceState *st = &g_static_state[device];
+    std::lock_guard<std::mutex> lock(g_static_mutex);
     if (!st->ready) {
         if (cudaDeviceGetAttribute(&cc, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
             cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
@@ -432,10 +427,10 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     int32_t *status = (int32_t *)st->scratch;
     float4 *partials = (float4 *)(st->scratch + kStaticHeaderBytes);
     // The array keeps the previous call's contents.  The status word must start at zero; the partial
-    // states need no clearing: the GEMM kernel writes every (row, range) entry the merge kernel reads.
+    // states need no clearing: the projection kernel writes every (row, range) entry the merge kernel reads.
     if (cudaMemsetAsync(status, 0, sizeof(int32_t), s) != cudaSuccess) return PVF_ERR_CUDA;
-    return launch_score(g, hidden, M, vocab, hidden_size, w_levels, partials, status, plan_bitmap, tok, conf, ent,
-                        in_plan, s, nullptr, nullptr);
+    if ((rc = launch_projection(g, hidden, M, vocab, hidden_size, w_levels, partials, status, s, nullptr, nullptr)) != PVF_OK) return rc;
+    return launch_merge(partials, M, g.parts, vocab, plan_bitmap, tok, conf, ent, in_plan, s);
 }
 
 int pvf_score_static_status(int32_t *status)
@@ -444,8 +439,43 @@ int pvf_score_static_status(int32_t *status)
     StaticDeviceState *st = nullptr;
     int rc = static_device_state(&st);
     if (rc != PVF_OK) return rc;
-    if (cudaMemcpy(status, st->scratch, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess) return PVF_ERR_CUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess ||       // every stream of the device, non-blocking ones included
+        cudaMemcpy(status, st->scratch, sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return PVF_ERR_CUDA;
     return PVF_OK;
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------- self-test of the bounded wait
+// Not part of the C interface (not declared in pvf.h): exercises, in its harmless form, the path every kernel takes
+// when a wait runs out.  One small block initialises an mbarrier that nothing ever arrives on and waits on it with
+// the projection kernels' own bounded wait and a caller-given limit; no copy, no MMA and no tensor memory is in
+// flight.  The wait gives up, the status word receives PVF_ERR_TIMEOUT, the kernel returns and the context stays usable.
+namespace {
+
+__global__ void __launch_bounds__(64)
+pvf_wait_expiry_kernel(int32_t *status, unsigned long long limit_ns, int32_t *gave_up)
+{
+    __shared__ SharedControl ctl;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&ctl.full[0]), 1);
+        ctl.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    bool ok = true;
+    if (threadIdx.x == 0) ok = mbar_wait_slow(smem_u32(&ctl.full[0]), 0u, &ctl, status, limit_ns);     // runs out
+    __syncthreads();
+    if (threadIdx.x == 32) ok = mbar_wait_slow(smem_u32(&ctl.full[0]), 0u, &ctl, status, limit_ns);    // sees the abort flag
+    if ((threadIdx.x == 0 || threadIdx.x == 32) && !ok) atomicAdd(gave_up, 1);
+}
+
+}  // namespace
+
+extern "C" int pvf_selftest_wait_expiry(pvf_ctx *ctx, uint64_t limit_ns, int32_t *gave_up, void *stream)
+{
+    if (!ctx || !gave_up || limit_ns == 0 || limit_ns > 100000000ull) return PVF_ERR_INVALID;   // at most 0.1 s
+    pvf_wait_expiry_kernel<<<1, 64, 0, (cudaStream_t)stream>>>(&ctx->words->status, (unsigned long long)limit_ns, gave_up);
+    return cudaGetLastError() == cudaSuccess ? PVF_OK : PVF_ERR_CUDA;
+}

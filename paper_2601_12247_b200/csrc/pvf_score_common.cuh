@@ -7,40 +7,19 @@
 #include "pvf_internal.h"
 
 
-// Tile shapes (overridable at build time for tuning sweeps).
-#ifndef PVF_STREAM_STAGES
-#define PVF_STREAM_STAGES 6
-#endif
-#ifndef PVF_GENERAL_TILE_N
-#define PVF_GENERAL_TILE_N 256
-#endif
-#ifndef PVF_GENERAL_PANELS
-#define PVF_GENERAL_PANELS 1
-#endif
-#ifndef PVF_GENERAL_STAGES
-#define PVF_GENERAL_STAGES 4
-#endif
-#ifndef PVF_PAIR_MIN_TILES
-#define PVF_PAIR_MIN_TILES 2     // 128-row tiles from which the paired (cta_group::2) kernel takes over
-#endif
-#ifndef PVF_PAIR_MAX_ROWS
-#define PVF_PAIR_MAX_ROWS 8192   // rows up to which the paired kernel is considered
-#endif
-#ifndef PVF_SWAP_SMALL_MAX_ROWS
-#define PVF_SWAP_SMALL_MAX_ROWS 64     // 33 .. this many rows take the swapped paired kernel
-#endif
-#ifndef PVF_SWAP_RAGGED_MAX_ROWS
-#define PVF_SWAP_RAGGED_MAX_ROWS 192   // and so do 129 .. this many rows (at most 256)
-#endif
-#ifndef PVF_SWAP_WIDE_WARPS
-#define PVF_SWAP_WIDE_WARPS 3          // epilogue warps per lane quadrant of the swapped paired kernel above 256 rows
-#endif
-#ifndef PVF_SWAP_WIDE_MAX_ROWS
-#define PVF_SWAP_WIDE_MAX_ROWS 448     // and 257 .. this many rows (at most 512; 0 = never), in two column groups
-#endif
-
 namespace {
 
+
+// Tile shapes and the row windows of the four kernels (settled by measurement).
+constexpr int kGeneralTileN = 256;         // 128-row GEMM kernel: vocabulary entries per accumulator
+constexpr int kGeneralPanels = 1;          //   64-element k-panels per pipeline stage
+constexpr int kGeneralStages = 4;          //   pipeline stages
+constexpr int kPairMinTiles = 2;           // 128-row tiles from which the paired (cta_group::2) kernel takes over
+constexpr int kPairMaxRows = 8192;         // rows up to which the paired kernel is considered
+constexpr int kSwapSmallMaxRows = 64;      // 33 .. this many rows take the swapped paired kernel
+constexpr int kSwapRaggedMaxRows = 192;    // and so do 129 .. this many rows (at most 256)
+constexpr int kSwapWideWarps = 3;          // epilogue warps per lane quadrant of the swapped paired kernel above 256 rows
+constexpr int kSwapWideMaxRows = 448;      // and 257 .. this many rows (at most 512), in two column groups
 
 constexpr int kTileM = 128;                // rows per accumulator (tensor-memory lanes)
 constexpr int kUnit = 16;                  // vocabulary granule
@@ -72,7 +51,7 @@ struct GemmCfg {
     static_assert(kSmemBytes <= 227 * 1024, "shared memory");
 };
 
-using GeneralCfg = GemmCfg<PVF_GENERAL_TILE_N, PVF_GENERAL_PANELS, PVF_GENERAL_STAGES>;
+using GeneralCfg = GemmCfg<kGeneralTileN, kGeneralPanels, kGeneralStages>;
 
 struct __align__(8) SharedControl {
     unsigned long long full[kMaxStages];   // TMA bytes landed
@@ -100,6 +79,7 @@ struct ScoreArgs {
     int m_tiles, mb, splits, waves;
     int a_rows;          // rows per H box
     int n_pad, stages;   // swapped paired kernel: rows per row tile (MMA N), pipeline stages
+    int w_once;          // 1: the launch reads every W tile exactly once (its L2 lines are marked evict-first)
     int parts;           // partial states per row (row stride of `partials`)
     float4 *partials;    // [M][parts]
     int32_t *status;
@@ -138,14 +118,15 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 }
 
 // Bounded wait.  Returns false when the block is aborting (this wait ran out, or another did).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, SharedControl *ctl, int32_t *status)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, SharedControl *ctl, int32_t *status,
+                                            unsigned long long limit_ns = kWaitLimitNs)
 {
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (ctl->abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
+        if (global_timer_ns() - t0 > limit_ns) {
             ctl->abort_flag = 1;
             atomicExch(status, (int32_t)PVF_ERR_TIMEOUT);
             return false;
@@ -163,6 +144,24 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+
+// L2 eviction priority for the W tiles.  Where a launch reads W exactly once (one wave, one row tile in flight) the
+// tiles are marked evict-first: a gigabyte of weights then streams through L2 without pushing out what the small
+// kernels behind the projection need (their instructions, the partial states, the hidden states); where blocks share W
+// tiles through L2 (several row tiles in flight) the priority stays normal.
+__device__ __forceinline__ uint64_t w_l2_policy(int read_once)
+{
+    uint64_t p;
+    if (read_once) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -217,11 +216,27 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
-__device__ __forceinline__ float fast_exp2(float x)
+__device__ __forceinline__ float fast_exp2(float x) { return pvf_fast_exp2(x); }
+
+// Bounded wait (no more than kWaitLimitNs) until the copies a producer thread armed on full[0 .. stages) have
+// landed: the abort path's drain, so that no copy is in flight into shared memory that is about to be released.
+// The producer keeps two bit sets (registers, no local memory): bit s of `armed` is set once full[s] has been armed,
+// bit s of `parity` is the phase parity the barrier had when it was last armed.
+struct ArmedStages {
+    uint32_t armed = 0, parity = 0;
+    __device__ __forceinline__ void note(int stage, uint32_t phase)
+    {
+        armed |= 1u << stage;
+        parity = (parity & ~(1u << stage)) | (phase << stage);
+    }
+};
+__device__ __forceinline__ void drain_armed_stages(SharedControl *ctl, const ArmedStages &a, int stages)
 {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
+    for (int s = 0; s < stages; ++s)
+        if ((a.armed >> s) & 1u) {
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(smem_u32(&ctl->full[s]), (a.parity >> s) & 1u) && global_timer_ns() - t0 < kWaitLimitNs) {}
+        }
 }
 
 // Barrier set-up shared by the three projection kernels (one thread): `issuers` threads commit every stage and
@@ -280,7 +295,7 @@ struct TileSplit {
 // kept OUT of the sum: beside it, the other terms of a peaked row (e^-17 = 4e-8 each, a hundred thousand of them,
 // half a per cent of the mass together) lie below the fp32 rounding unit of 1.0 and would be rounded away one by
 // one.  The row's normaliser is 1 + s.  The state is empty while arg is kNoArg.
-constexpr int kNoArg = 0x7fffffff;
+constexpr int kNoArg = kPvfNoArg;
 struct RowState {
     float m;      // running max
     float s;      // sum of e^{x - m} over every column except the one that holds the max
@@ -328,10 +343,11 @@ __device__ __forceinline__ void fold16(RowState &st, const uint32_t (&raw)[16], 
     st.s += group;
 }
 
+
 // One W tile of `tun` granules starting at granule tu0, columns x .. x+63, into b_dst.
-__device__ __forceinline__ void load_w_tile(uint32_t b_dst, const WMaps &maps, uint32_t full, int x, int tu0, int tun)
+__device__ __forceinline__ void load_w_tile(uint32_t b_dst, const WMaps &maps, uint32_t full, int x, int tu0, int tun, uint64_t policy)
 {
-    tma_load_2d(b_dst, &maps.size[tun - 1], full, x, tu0 * kUnit);
+    tma_load_2d_hint(b_dst, &maps.size[tun - 1], full, x, tu0 * kUnit, policy);
 }
 
 }  // namespace

@@ -55,9 +55,8 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            int armed_parity[kStages];
-#pragma unroll
-            for (int s = 0; s < kStages; ++s) armed_parity[s] = -1;
+            ArmedStages armed;
+            const uint64_t w_policy = w_l2_policy(args.w_once);
             bool alive = true;
             for (int w = 0; w < args.waves && alive; ++w) {
                 const int m_tile = w * args.mb + mt_local;
@@ -74,25 +73,18 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
                         const uint32_t a_base = tiles_addr + stage * Cfg::kStageBytes;
                         const uint32_t b_base = a_base + kPanels * Cfg::kAPanelBytes;
                         mbar_arrive_expect_tx(full, panel_bytes * (uint32_t)np);
-                        armed_parity[stage] = (int)phase;
+                        armed.note(stage, phase);
                         for (int p = 0; p < np; ++p) {
                             const int x = (kb0 + p) * kBlockK;
                             tma_load_2d(a_base + p * Cfg::kAPanelBytes, &tm_h, full, x, m_tile * kTileM);
-                            load_w_tile(b_base + p * Cfg::kBPanelBytes, tm_w, full, x, tu0, tun);
+                            load_w_tile(b_base + p * Cfg::kBPanelBytes, tm_w, full, x, tu0, tun, w_policy);
                         }
                         if (++stage == kStages) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
-            if (!alive) {
-                // Abort: let every copy this thread started land before the block's memory is released.
-                for (int s = 0; s < kStages; ++s)
-                    if (armed_parity[s] >= 0) {
-                        const unsigned long long t0 = global_timer_ns();
-                        while (!mbar_try_wait(smem_u32(&ctl->full[s]), (uint32_t)armed_parity[s]) &&
-                               global_timer_ns() - t0 < kWaitLimitNs) {}
-                    }
-            }
+            // Abort: let every copy this thread started land before the block's memory is released.
+            if (!alive) drain_armed_stages(ctl, armed, kStages);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer

@@ -49,6 +49,12 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"((unsigned long long)map), "r"(bar & kPeerBitMask), "r"(x), "r"(y) : "memory");
 }
+__device__ __forceinline__ void tma_load_2d_pair_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"((unsigned long long)map), "r"(bar & kPeerBitMask), "r"(x), "r"(y), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                                  uint32_t accumulate)
 {
@@ -123,6 +129,8 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
+            ArmedStages armed;
+            const uint64_t w_policy = w_l2_policy(args.w_once);
             bool alive = true;
             for (int w = 0; w < args.waves && alive; ++w) {
                 const int s_tile = w * args.mb + st_local;
@@ -137,17 +145,23 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
                         if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
                         const uint32_t full = smem_u32(&ctl->full[stage]);
                         const uint32_t a_dst = tiles_addr + stage * kPairStageBytes;
-                        if (rank == 0) mbar_arrive_expect_tx(full, bytes);
+                        if (rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
                         tma_load_2d_pair(a_dst, &tm_h, full, step * kBlockK, row0);
-                        tma_load_2d_pair(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
+                        tma_load_2d_pair_hint(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
                         if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
                     }
                 }
             }
             if (!alive) {
-                // Abort: give the copies in flight time to land before the pair leaves.
-                const unsigned long long t0 = global_timer_ns();
-                while (global_timer_ns() - t0 < 200000ull) {}
+                // Abort: the copies in flight land before the pair leaves.  The even block's full[] barriers count
+                // both blocks' bytes, so it waits (bounded) on every stage it armed; the odd block has no barrier
+                // of its own to wait on and gives its copies a fixed time (the closing cluster barrier holds both
+                // blocks until the slower one is through).
+                if (rank == 0) drain_armed_stages(ctl, armed, kPairStages);
+                else {
+                    const unsigned long long t0 = global_timer_ns();
+                    while (global_timer_ns() - t0 < 200000ull) {}
+                }
             }
         }
     } else if (warp == 1) {

@@ -16,7 +16,7 @@ namespace {
 // now owns a vocabulary lane: it keeps one running softmax state per scored row (for the vocabulary
 // entries that passed through its lane) and the block folds the 128 lanes' states once, at the end,
 // through shared memory.  The per-(row, range) partial state it leaves is the GEMM kernel's.
-constexpr int kStreamStages = PVF_STREAM_STAGES;
+constexpr int kStreamStages = 6;
 constexpr int kStreamTileN = 256;                                   // vocabulary entries per W tile (two 128-lane slices)
 constexpr int kStreamUnitsPerTile = kStreamTileN / kUnit;
 constexpr int kStreamHBytes = kStreamRows * kRowBytes;              // 4 KiB
@@ -52,31 +52,6 @@ __device__ __forceinline__ void state_push(float &m, float &s, float &t, int &ar
         const float e = fast_exp2(d * kLog2e);
         s += e;
         t = fmaf(d, e, t);
-    }
-}
-
-// a <- a merged with b (two states over disjoint vocabulary sets).  The larger max stays outside the sum; the
-// other state's max joins it as an ordinary term.
-__device__ __forceinline__ void state_merge(float4 &a, const float4 b)
-{
-    constexpr float kLog2e = 1.4426950408889634f;
-    const int ia = __float_as_int(a.w), ib = __float_as_int(b.w);
-    if (ib == kNoArg) return;
-    if (ia == kNoArg) { a = b; return; }
-    if (a.x > b.x || (a.x == b.x && ia < ib)) {
-        const float d = b.x - a.x;                      // <= 0
-        const float c = fast_exp2(d * kLog2e);
-        const float total = b.y + 1.f;
-        a.y += total * c;
-        a.z += (b.z + d * total) * c;
-    } else {
-        const float d = a.x - b.x;
-        const float c = fast_exp2(d * kLog2e);
-        const float total = a.y + 1.f;
-        a.y = b.y + total * c;
-        a.z = b.z + (a.z + d * total) * c;
-        a.x = b.x;
-        a.w = b.w;
     }
 }
 
@@ -120,9 +95,8 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            int armed_parity[kStreamStages];
-#pragma unroll
-            for (int s = 0; s < kStreamStages; ++s) armed_parity[s] = -1;
+            ArmedStages armed;
+            const uint64_t w_policy = w_l2_policy(args.w_once);
             bool alive = true;
             for (int tile = 0; tile < n_tiles && alive; ++tile) {
                 int tu0, tun;
@@ -133,20 +107,13 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     const uint32_t h_dst = tiles_addr + stage * kStreamStageBytes;
                     mbar_arrive_expect_tx(full, bytes);
-                    armed_parity[stage] = (int)phase;
+                    armed.note(stage, phase);
                     tma_load_2d(h_dst, &tm_h, full, step * kBlockK, 0);
-                    load_w_tile(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun);
+                    load_w_tile(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, w_policy);
                     if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
                 }
             }
-            if (!alive) {
-                for (int s = 0; s < kStreamStages; ++s)
-                    if (armed_parity[s] >= 0) {
-                        const unsigned long long t0 = global_timer_ns();
-                        while (!mbar_try_wait(smem_u32(&ctl->full[s]), (uint32_t)armed_parity[s]) &&
-                               global_timer_ns() - t0 < kWaitLimitNs) {}
-                    }
-            }
+            if (!alive) drain_armed_stages(ctl, armed, kStreamStages);
         }
     } else if (warp == 1 || warp == kStreamSecondIssuerWarp) {
         // ------------------------------------------------------------------ MMA issuers
@@ -250,14 +217,14 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
             const int e = threadIdx.x - 64;                              // 0..127
             const int row = e >> 2, part = e & 3;
             float4 acc = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(kNoArg));
-            for (int l = 0; l < 32; ++l) state_merge(acc, scratch[row * kTileM + part * 32 + l]);
+            for (int l = 0; l < 32; ++l) pvf_state_merge(acc, scratch[row * kTileM + part * 32 + l]);
             for (int o = 1; o < 4; o <<= 1) {
                 float4 other;
                 other.x = __shfl_xor_sync(0xffffffffu, acc.x, o);
                 other.y = __shfl_xor_sync(0xffffffffu, acc.y, o);
                 other.z = __shfl_xor_sync(0xffffffffu, acc.z, o);
                 other.w = __shfl_xor_sync(0xffffffffu, acc.w, o);
-                state_merge(acc, other);
+                pvf_state_merge(acc, other);
             }
             if (part == 0 && row < args.M) args.partials[(size_t)row * args.splits + q] = acc;
         }

@@ -28,7 +28,7 @@ namespace {
 // k-step (one loop serving one or two column groups) cost 17 .. 33 % of the whole launch; the two cases are
 // separate loops.
 //
-// Epilogue: one warp per quadrant of 32 vocabulary lanes up to 256 rows, PVF_SWAP_WIDE_WARPS above, taking the
+// Epilogue: one warp per quadrant of 32 vocabulary lanes up to 256 rows, kSwapWideWarps above, taking the
 // groups of 32 rows (columns) in turn.  A warp turns its 32 x 32 block
 // around through a padded shared-memory tile of its own, after which lane i holds row i's 32 logits and folds
 // them into the running state of row chunk*32 + i exactly as the GEMM kernels' epilogue does (no warp-wide
@@ -41,22 +41,22 @@ constexpr int kSwapWBytes = kTileM * kRowBytes;                      // 16 KiB
 constexpr int kSwapGroupCols = 256;                                  // MMA N limit: columns (rows of H) per MMA
 constexpr int kSwapMaxRows = 512;                                    // two column groups fill tensor memory
 constexpr int kSwapTmemCols = 512;                                   // two accumulators of up to 256 columns, or one of up to 512
-constexpr int kSwapEpilogueWarps = 4 * PVF_SWAP_WIDE_WARPS;          // at most; one per tensor-memory lane quadrant works on up to
-                                                                     // 256 rows, PVF_SWAP_WIDE_WARPS (taking row chunks in turn) above
+constexpr int kSwapEpilogueWarps = 4 * kSwapWideWarps;          // at most; one per tensor-memory lane quadrant works on up to
+                                                                     // 256 rows, kSwapWideWarps (taking row chunks in turn) above
 constexpr int kSwapEpilogueThreads = kSwapEpilogueWarps * 32;
 constexpr int kSwapThreads = 64 + kSwapEpilogueThreads;              // producer warp, MMA warp, epilogue warps
 constexpr int kSwapTurnPitch = 33;                                   // words per lane of a warp's 32 x 32 fp32 block (conflict-free both ways)
 constexpr int kSwapWarpScratchBytes = 32 * kSwapTurnPitch * 4;       // that block, one per epilogue warp
 // Scratch of one quadrant = its warps' blocks; at the end it holds the quadrant's row states (16 bytes per row).
-__host__ __device__ constexpr int swap_warps_per_quad(int n_pad) { return n_pad > kSwapGroupCols ? PVF_SWAP_WIDE_WARPS : 1; }
+__host__ __device__ constexpr int swap_warps_per_quad(int n_pad) { return n_pad > kSwapGroupCols ? kSwapWideWarps : 1; }
 __host__ __device__ constexpr int swap_quad_scratch_bytes(int n_pad) { return swap_warps_per_quad(n_pad) * kSwapWarpScratchBytes; }
 constexpr int kSwapMaxStages = 12;
 constexpr int kSwapSmemBytes = 227 * 1024;                           // everything: alignment slack, ring, control block, scratch
 static_assert(swap_quad_scratch_bytes(kSwapMaxRows) >= kSwapMaxRows * 16 && swap_quad_scratch_bytes(kSwapGroupCols) >= kSwapGroupCols * 16 &&
               kSwapWarpScratchBytes % 16 == 0, "fold scratch");
 static_assert(kSwapMaxStages <= kMaxStages, "barrier arrays");
-static_assert(PVF_SWAP_SMALL_MAX_ROWS <= kSwapGroupCols && PVF_SWAP_RAGGED_MAX_ROWS <= kSwapGroupCols &&
-              PVF_SWAP_WIDE_MAX_ROWS <= kSwapMaxRows, "row limits");
+static_assert(kSwapSmallMaxRows <= kSwapGroupCols && kSwapRaggedMaxRows <= kSwapGroupCols &&
+              kSwapWideMaxRows <= kSwapMaxRows, "row limits");
 
 __host__ __device__ constexpr int swap_stage_bytes(int n_pad) { return kSwapWBytes + (n_pad / 2) * kRowBytes; }
 // Pipeline stages that fit beside the control block and the epilogue's scratch.
@@ -71,7 +71,7 @@ inline int swap_stages(int n_pad)
 // two threads set the pace of the kernel, and a run-time choice inside their loops costs more than it looks.
 struct SwapLoopArgs {
     uint32_t tiles_addr, stage_bytes, h0_bytes, h1_bytes, tmem_base;
-    int n0, n1, n_stages, n_tiles, k_steps, n_bufs;
+    int n0, n1, n_stages, n_tiles, k_steps, n_bufs, w_once;
     uint32_t rank;
 };
 
@@ -83,6 +83,8 @@ __device__ __forceinline__ void swap_produce(const SwapLoopArgs &a, const TileSp
     int stage = 0;
     uint32_t phase = 0;
     bool alive = true;
+    ArmedStages armed;
+    const uint64_t w_policy = w_l2_policy(a.w_once);
     const int row0 = (int)a.rank * (a.n0 / 2);                                      // this block's half of each group's rows
     const int row1 = a.n0 + (int)a.rank * (a.n1 / 2);
     for (int tile = 0; tile < a.n_tiles && alive; ++tile) {
@@ -94,17 +96,21 @@ __device__ __forceinline__ void swap_produce(const SwapLoopArgs &a, const TileSp
             if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, status)) { alive = false; break; }
             const uint32_t full = smem_u32(&ctl->full[stage]);
             const uint32_t w_dst = a.tiles_addr + (uint32_t)stage * a.stage_bytes;
-            if (a.rank == 0) mbar_arrive_expect_tx(full, bytes);
-            tma_load_2d_pair(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
+            if (a.rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
+            tma_load_2d_pair_hint(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
             tma_load_2d_pair(w_dst + kSwapWBytes, tm_h, full, step * kBlockK, row0);
             if (kWide) tma_load_2d_pair(w_dst + kSwapWBytes + a.h0_bytes, tm_h1, full, step * kBlockK, row1);
             if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
         }
     }
     if (!alive) {
-        // Abort: give the copies in flight time to land before the pair leaves.
-        const unsigned long long t0 = global_timer_ns();
-        while (global_timer_ns() - t0 < 200000ull) {}
+        // Abort: the copies in flight land before the pair leaves (see the paired GEMM kernel: the even block waits,
+        // bounded, on the barriers it armed; the odd block gives its copies a fixed time).
+        if (a.rank == 0) drain_armed_stages(ctl, armed, a.n_stages);
+        else {
+            const unsigned long long t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 200000ull) {}
+        }
     }
 }
 
@@ -208,7 +214,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     SwapLoopArgs la;
     la.tiles_addr = tiles_addr; la.stage_bytes = stage_bytes; la.h0_bytes = h0_bytes; la.h1_bytes = h1_bytes;
     la.tmem_base = tmem_base; la.n0 = n0; la.n1 = n1; la.n_stages = n_stages; la.n_tiles = n_tiles; la.k_steps = k_steps;
-    la.n_bufs = n_bufs; la.rank = rank;
+    la.n_bufs = n_bufs; la.rank = rank; la.w_once = args.w_once;
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (one per block)
         if (lane == 0) {
@@ -298,7 +304,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
                 float4 acc = reinterpret_cast<const float4 *>(scratch)[row];
 #pragma unroll
                 for (int o = 1; o < 4; ++o)
-                    state_merge(acc, reinterpret_cast<const float4 *>(scratch + o * quad_scratch)[row]);
+                    pvf_state_merge(acc, reinterpret_cast<const float4 *>(scratch + o * quad_scratch)[row]);
                 args.partials[(size_t)row * args.parts + 2 * q + (int)rank] = acc;
             }
         }

@@ -5,10 +5,10 @@ the scored rows are re-drawn on the host from (seed, step, sequence, position), 
 grows with the sequence's committed fraction, and uploaded.  Decoding is semi-autoregressive: the
 working block of a sequence is its first block that still holds a mask; the scored rows are that block's
 masked positions, widened by the next block under early cross-block revelation (``n_sparse``); the rows
-come from pvf_working_set on the device.  One step = draft-pass score, commit, draft selection, verification-pass score, verify;
-it counts as one batched forward.  ``budget = 0`` gives confidence-threshold decoding.
+come from pvf_working_set on the device.  One step = pvf_draft_step (draft-pass score, base commit and draft selection) and
+pvf_verify_step (verification-pass score, verify); it counts as one batched forward.  ``budget = 0`` gives confidence-threshold decoding.
 
-This is a harness around the library (the hot path is the five kernels); it reports steps,
+This is a harness around the library (the hot path is the library's kernels); it reports steps,
 tokens per forward, scored rows and the kernel time per step measured with CUDA events.
 
     python -m paper_2601_12247_b200.decode_loop [--n-seq 32] [--gen-len 256] [--block 32] [--budget 4]
@@ -56,16 +56,21 @@ def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: 
         seg, pos = ws["seg_off"], ws["row_pos"][:n_rows]
         e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         e[0].record()
-        sc = ctx.score(h)
-        cm = ctx.commit(prm, seg, pos, None, sc["tok"], sc["conf"], y=y_dev)
         sel = ver = scv = exp_row = None
         hv_bits = None
+        if K > 0 and not explore:
+            # score, then base commit and draft proposal in one launch
+            d = ctx.draft_step(prm, h, seg, pos, None, y=y_dev)
+            sc = {k: d[k] for k in ("tok", "conf", "ent", "in_plan")}
+            cm = {k: d[k] for k in ("commit", "n_commit")}
+            sel = {k: d[k] for k in ("draft_rows", "n_drafts", "route", "rem_rows", "rem_off", "v_off")}
+        else:
+            sc = ctx.score(h)
+            cm = ctx.commit(prm, seg, pos, None, sc["tok"], sc["conf"], y=y_dev)
         if explore:
             u = torch.from_numpy(synth.loop_uniforms(seed, n_steps, n_seq)).to(dev)
             mode = binding.PVF_EXPLORE_PLANNING if explore == "planning" else binding.PVF_EXPLORE_RANDOM
             exp_row = ctx.explore_commit(prm, mode, seg, pos, None, sc["tok"], sc["conf"], sc["in_plan"], u, cm["commit"], y=y_dev)
-        if K > 0:
-            sel = ctx.select_drafts(prm, seg, pos, None, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
         e[1].record()
         scored_rows += len(positions)
         if K > 0:
@@ -82,8 +87,9 @@ def decode(ctx: binding.Context, w_bits: np.ndarray, targets: np.ndarray, seed: 
             hv_bits = synth.loop_verify_hidden(w_bits, targets, seed, n_steps, vb, vi, vc, frac)
             hv = binding.bf16_from_bits(hv_bits, dev)
             e[2].record()
-            scv = ctx.score(hv)
-            ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"], y=y_dev)
+            vs = ctx.verify_step(prm, hv, seg, pos, d, y=y_dev)
+            scv = dict(tok=vs["tok_v"], conf=vs["conf_v"], ent=vs["ent_v"])
+            ver = {k: vs[k] for k in ("accept", "choice", "final_commit")}
             e[3].record()
             scored_rows += len(vb)
         torch.cuda.synchronize()

@@ -40,7 +40,7 @@ def test_default_workload_line():
     assert cfg["workload"] == "cfg1a" and cfg["draft_rows"] == 32 and "model" not in cfg
     # value = draft rows per second of the whole step
     assert d["value"] == pytest.approx(cfg["draft_rows"] / (d["ms_per_step"] * 1e-3), rel=1e-6)
-    assert d["gpu_launches"] == 7 * d["steps"]                      # 2 x (projection + merge) + commit + select + verify
+    assert d["gpu_launches"] == 4 * d["steps"]                      # 2 x projection (merge in its tail) + commit_select + verify
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["kernel"] == "pvf_score_stream_kernel"
     assert r["frac"] == pytest.approx(r["achieved"] / r["peak"], rel=1e-9)
@@ -88,9 +88,9 @@ def test_tensor_regime_launch_times_fit_their_step():
     d = run_bench("--workload", "cfg3s", "--steps", "4", "--warmup", "3", "--min-seconds", "1", "--no-cpu-baseline", "--no-graph")
     r = d["roofline"]
     assert r["bound"] == "tensor" and r["timed_every_nth_step"] == 1 and d["config"]["draft_rows"] == 4096
-    assert r["launches"] == 2 * d["steps"] * d["repeats"]
+    assert r["launches"] == 2 * d["steps"] and d["repeats"] >= 3      # the median block's own launches
     launches_fit_the_step(r, d["ms_per_step"])
-    assert d["gpu_launches"] == 7 * d["steps"]
+    assert d["gpu_launches"] == 4 * d["steps"]
 
 
 def test_ridge_workload_reports_the_kernel_mix():
@@ -98,4 +98,4 @@ def test_ridge_workload_reports_the_kernel_mix():
     r = d["roofline"]
     assert set(r["kernel"].split("+")) == {"pvf_score_gemm_pair_kernel", "pvf_score_swap_pair_kernel"}
     assert d["config"]["draft_rows"] == 232 and d["config"]["verify_rows"] == 181
-    assert r["traffic"] is not None and d["gpu_launches"] == 7 * d["steps"]
+    assert r["traffic"] is not None and d["gpu_launches"] == 4 * d["steps"]

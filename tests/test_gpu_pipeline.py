@@ -118,6 +118,65 @@ def test_config2_and_3_at_small_vocab(stress):
     ctx.close()
 
 
+@pytest.mark.parametrize("force", [0, binding.PVF_FORCE_PROGRESS])
+def test_step_calls_equal_the_four_calls(force):
+    # pvf_draft_step / pvf_verify_step (two launches each) against pvf_score, pvf_commit, pvf_select_drafts, pvf_verify
+    # called one by one: the same kernels on the same inputs, so every output is bit-identical, canvas included
+    w = synth.make_w(2002, 8192, 256)
+    st = synth.config2(stress=True, w_bits=w, vocab=8192, hidden=256)
+    ctx = make_ctx(w, st.plan_ids, 8192, 64, 16)
+    prm = params_of(st, force, tau_high=0.97 if force else st.params["tau_high"])
+    seg, pos, act = t_i32(st.seg_off), t_i32(st.row_pos), t_u8(st.active)
+    h = upload_bits(st.h_bits)
+    y_a = torch.full((st.n_seq, st.gen_len), -1, dtype=torch.int32, device=dev())
+    y_b = y_a.clone()
+    sc = ctx.score(h)
+    cm = ctx.commit(prm, seg, pos, act, sc["tok"], sc["conf"], y=y_a)
+    sel = ctx.select_drafts(prm, seg, pos, act, sc["tok"], sc["conf"], sc["in_plan"], cm["commit"])
+    d = ctx.draft_step(prm, h, seg, pos, act, y=y_b)
+    torch.cuda.synchronize()
+    one, two = dict(to_np(sc), **to_np(cm), **to_np(sel)), to_np(d)
+    n_rem = int(one["rem_off"][-1])
+    for k in one:
+        a, b = (one[k][:n_rem], two[k][:n_rem]) if k == "rem_rows" else (one[k], two[k])
+        assert np.array_equal(a.view(np.uint8), b.view(np.uint8)), k
+    assert torch.equal(y_a, y_b)
+    v = synth.make_verify_pass(st, one["rem_rows"][:n_rem], one["rem_off"], one["n_drafts"])
+    assert v.hv_bits.shape[0] > 0
+    hv = upload_bits(v.hv_bits)
+    scv = ctx.score(hv)
+    ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"], y=y_a)
+    vs = ctx.verify_step(prm, hv, seg, pos, d, y=y_b)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    assert torch.equal(scv["tok"], vs["tok_v"]) and torch.equal(scv["conf"].view(torch.int32), vs["conf_v"].view(torch.int32))
+    for k in ("accept", "choice", "final_commit"):
+        assert torch.equal(ver[k], vs[k]), k
+    assert torch.equal(y_a, y_b) and (to_np(ver)["choice"] > 0).any()
+    ctx.close()
+
+
+def test_scores_are_identical_from_run_to_run():
+    # the tail's merge is done by whichever block finishes last, in an order fixed by the data layout alone: repeated
+    # calls give the same bits, for every kernel (row counts of the streaming, swapped, 128-row and paired kernels)
+    w = synth.make_w(2003, 20000, 512)
+    pos = np.arange(600)
+    st = synth.build_step("repeat", 2003, 20000, 512, 256, [(pos, np.ones(600, np.uint8))], 600, 600,
+                          dict(tau_high=0.9, budget=4), stress=True, w_bits=w)
+    ctx = make_ctx(w, st.plan_ids, 1024)
+    kernels = set()
+    for rows in (24, 60, 100, 170, 256, 300, 600):
+        h = upload_bits(st.h_bits[:rows])
+        kernels.add(ctx.score_kernel_name(rows))
+        first = to_np(ctx.score(h))
+        for _ in range(5):
+            again = to_np(ctx.score(h))
+            for k in first:
+                assert np.array_equal(first[k].view(np.uint8), again[k].view(np.uint8)), (rows, k)
+    assert len(kernels) == 4 and ctx.last_status() == 0
+    ctx.close()
+
+
 # ------------------------------------------------------------------------------ LLaDA shape
 @pytest.fixture(scope="module")
 def llada():

@@ -57,6 +57,14 @@ def run_step(ctx, c, tau_high=0.9, flags=0, rng=None, agree=0.7):
     for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
         assert np.array_equal(gs[k], osel[k]), k
     assert np.array_equal(gs["rem_rows"][:n_rem], osel["rem_rows"])
+    # the fused call (one launch) gives what the two calls gave, bit for bit, canvas included
+    y2 = t_i32(y0)
+    both = to_np(ctx.commit_select(prm, seg, pos, act, tok, conf, inp, y=y2))
+    assert np.array_equal(both["commit"], g["commit"]) and np.array_equal(both["n_commit"], g["n_commit"])
+    assert np.array_equal(y2.cpu().numpy(), ocm["y"])
+    for k in ("draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+        assert np.array_equal(both[k], gs[k]), k
+    assert np.array_equal(both["rem_rows"][:n_rem], osel["rem_rows"])
 
     # verification-pass outputs: start from "every branch repeats the draft-pass token", then flip some
     rng = rng or np.random.default_rng(0)
