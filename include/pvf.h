@@ -133,14 +133,17 @@ int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int3
  * NULL) receives 0 for the streaming kernel, 1 for the 128-row GEMM kernel, 2 for the paired kernel, 3 for the paired
  * kernel with swapped operands; `row_tiles` the number of row tiles (256 rows in the paired kernel, one tile of up
  * to 512 rows in the swapped paired kernel, else 128) and `tiles_per_wave` how many are in flight.  For kernels 2
- * and 3 `splits` counts pairs of thread blocks. */
+ * and 3 `splits` counts pairs of thread blocks.  The paired kernel's last wave may hold fewer tiles than the others
+ * and split each over more pairs: `last_wave_tiles` (0: every wave is full) and `last_wave_splits`. */
 int pvf_score_plan_for_shape(int32_t vocab, int32_t hidden, int32_t n_sm, int32_t M, int32_t *ctas, int32_t *splits,
-                             int32_t *waves, int32_t *kernel, int32_t *row_tiles, int32_t *tiles_per_wave);
+                             int32_t *waves, int32_t *kernel, int32_t *row_tiles, int32_t *tiles_per_wave,
+                             int32_t *last_wave_tiles, int32_t *last_wave_splits);
 
 /* Name of the projection kernel pvf_score launches for M rows (for profiler filters and reports):
  * "pvf_score_stream_kernel" up to 32 rows (vocabulary on the accumulator lanes, rows on its columns),
  * "pvf_score_swap_pair_kernel" for 33 .. 64, 129 .. 192 and 257 .. 448 rows (the same layout, two thread blocks per
- * vocabulary tile), "pvf_score_gemm_kernel" or "pvf_score_gemm_pair_kernel" otherwise (rows on the lanes).
+ * vocabulary tile), "pvf_score_gemm_kernel" for 65 .. 128 rows and "pvf_score_gemm_pair_kernel" otherwise (rows on the
+ * lanes).
  * NULL on an invalid argument. */
 const char *pvf_score_kernel_name(pvf_ctx *ctx, int32_t M);
 

@@ -79,7 +79,7 @@ def load() -> ctypes.CDLL:
         lib.pvf_last_status.argtypes = [vp, ctypes.POINTER(i32)]; lib.pvf_last_status.restype = ctypes.c_int
         lib.pvf_set_score_events.argtypes = [vp, vp, vp]; lib.pvf_set_score_events.restype = ctypes.c_int
         lib.pvf_score_plan.argtypes = [vp, i32] + [ctypes.POINTER(i32)] * 4; lib.pvf_score_plan.restype = ctypes.c_int
-        lib.pvf_score_plan_for_shape.argtypes = [i32] * 4 + [ctypes.POINTER(i32)] * 6
+        lib.pvf_score_plan_for_shape.argtypes = [i32] * 4 + [ctypes.POINTER(i32)] * 8
         lib.pvf_score_plan_for_shape.restype = ctypes.c_int
         lib.pvf_score_kernel_name.argtypes = [vp, i32]; lib.pvf_score_kernel_name.restype = ctypes.c_char_p
         lib.pvf_score.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]; lib.pvf_score.restype = ctypes.c_int
@@ -125,10 +125,11 @@ def default_params() -> pvf_params:
 
 def score_plan_for_shape(vocab: int, hidden: int, n_sm: int, M: int) -> Dict[str, int]:
     """pvf_score_plan_for_shape: the work split pvf_score would use, computed on the host (no GPU needed)."""
-    v = [ctypes.c_int32() for _ in range(6)]
+    v = [ctypes.c_int32() for _ in range(8)]
     _check(load().pvf_score_plan_for_shape(int(vocab), int(hidden), int(n_sm), int(M), *[ctypes.byref(x) for x in v]),
            "pvf_score_plan_for_shape")
-    return dict(zip(("ctas", "splits", "waves", "kernel", "row_tiles", "tiles_per_wave"), (x.value for x in v)))
+    return dict(zip(("ctas", "splits", "waves", "kernel", "row_tiles", "tiles_per_wave", "last_wave_tiles", "last_wave_splits"),
+                    (x.value for x in v)))
 
 
 def default_calib_params() -> pvf_calib_params:

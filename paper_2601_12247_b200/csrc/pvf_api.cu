@@ -146,7 +146,7 @@ int pvf_last_status(pvf_ctx *ctx, int32_t *status)
     if (host != 0) {
         // A kernel gave up: clear the word (and the arrival tickets, which count whole blocks and so stay whole).
         if (cudaMemset(&ctx->words->status, 0, sizeof(int32_t)) != cudaSuccess ||
-            cudaMemset(&ctx->words->select_ticket, 0, 2 * sizeof(uint32_t)) != cudaSuccess ||
+            cudaMemset(&ctx->words->select_ticket, 0, 4 * sizeof(uint32_t)) != cudaSuccess ||
             cudaMemset(ctx->seq_tickets, 0, ctx->seq_tickets_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
             return PVF_ERR_CUDA;
     }

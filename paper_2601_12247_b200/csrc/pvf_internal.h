@@ -16,7 +16,9 @@ struct pvf_device_words {
     int32_t  status;        // PVF_OK or PVF_ERR_TIMEOUT, written by kernels
     uint32_t select_ticket; // blocks of pvf_select_drafts that have finished; reset by the last one
     uint32_t working_ticket; // the same for pvf_working_set
-    uint32_t pad[61];
+    uint32_t wave_arrivals; // paired projection kernel: blocks that have reached a wave boundary (all waves of a launch)
+    uint32_t wave_done;     //    blocks that are past their last wave boundary; the last one clears both
+    uint32_t pad[59];
 };
 
 struct pvf_ctx {
@@ -57,7 +59,10 @@ struct pvf_score_geometry {
                      //    granules of 32 entries, mb / splits pairs of blocks
     int n_pad;       // swapped: rows per row tile (multiple of 32, at most 256)
     int stages;      // swapped: pipeline stages that fit the shared-memory ring
-    int parts;       // partial states per row handed to the merge kernel (splits, or 2 * splits when swapped)
+    int parts;       // partial states per row handed to the merge kernel (splits, or 2 * splits when swapped; the
+                     //    larger of splits and splits_last when the last wave is split differently)
+    int mb_last;     // paired: row tiles of the last wave when it is a partial one (else 0), each swept by
+    int splits_last; //    splits_last pairs, so that the pairs are all busy in that wave too
 };
 // allow_swapped = false leaves the swapped paired kernel (which writes twice as many partial states per row) out.
 pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool allow_swapped = true);
@@ -96,22 +101,24 @@ static inline cudaError_t pvf_launch(void (*kernel)(KArgs...), dim3 grid, dim3 b
 // The same for a kernel whose blocks form clusters of two along x (grid.x even).
 template <typename... KArgs, typename... Args>
 static inline cudaError_t pvf_launch_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                              cudaStream_t stream, Args... args)
+                                              cudaStream_t stream, bool cooperative, Args... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[3];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[2].id = cudaLaunchAttributeCooperative;       // the launch fails unless every block can be resident at once
+    attr[2].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    cfg.numAttrs = cooperative ? 3 : 2;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif

@@ -124,7 +124,8 @@ int raise_shared_memory_limits()
 
 // Launches the projection kernel (shape chosen by the geometry) on `s`: it leaves g.parts partial states per row.
 int launch_projection(const pvf_score_geometry &g, const void *hidden, int M, int V, int D, const CUtensorMap *w_levels,
-                      float4 *partials, int32_t *status, cudaStream_t s, cudaEvent_t ev_start, cudaEvent_t ev_stop)
+                      float4 *partials, int32_t *status, uint32_t *wave_sync, cudaStream_t s, cudaEvent_t ev_start,
+                      cudaEvent_t ev_stop)
 {
     CUtensorMap tm_h;
     int rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)g.a_rows);
@@ -137,11 +138,13 @@ int launch_projection(const pvf_score_geometry &g, const void *hidden, int M, in
     a.num_kb = (D + kBlockK - 1) / kBlockK;
     a.units = g.units;
     a.m_tiles = g.m_tiles; a.mb = g.mb; a.splits = g.splits; a.waves = g.waves;
+    a.mb_last = g.mb_last; a.splits_last = g.splits_last;
     a.a_rows = g.a_rows;
     a.n_pad = g.n_pad; a.stages = g.stages; a.parts = g.parts;
     a.w_once = (g.waves == 1 && g.mb == 1) ? 1 : 0;
     a.partials = partials;
     a.status = status;
+    a.wave_sync = (g.paired && g.waves > 1) ? wave_sync : nullptr;
     const bool timed = ev_start && ev_stop;
     if (timed && cudaEventRecord(ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
     cudaError_t e;
@@ -150,10 +153,10 @@ int launch_projection(const pvf_score_geometry &g, const void *hidden, int M, in
         if (g.n_pad > kSwapGroupCols &&
             (rc = make_tensor_map(&tm_h1, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)((g.n_pad - kSwapGroupCols) / 2))) != PVF_OK)
             return rc;
-        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(64 + 128 * swap_warps_per_quad(g.n_pad)), kSwapSmemBytes, s, tm_h, tm_h1, maps, a);
+        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(64 + 128 * swap_warps_per_quad(g.n_pad)), kSwapSmemBytes, s, false, tm_h, tm_h1, maps, a);
     }
     else if (g.paired)
-        e = pvf_launch_cluster2(pvf_score_gemm_pair_kernel, dim3(g.ctas), dim3(kThreads), kPairSmemBytes, s, tm_h, maps, a);
+        e = pvf_launch_cluster2(pvf_score_gemm_pair_kernel, dim3(g.ctas), dim3(kThreads), kPairSmemBytes, s, a.wave_sync != nullptr, tm_h, maps, a);
     else if (g.streaming)
         e = pvf_launch(pvf_score_stream_kernel, dim3(g.ctas), dim3(kStreamThreads), kStreamSmemBytes, s, tm_h, maps, a);
     else
@@ -189,6 +192,7 @@ namespace {
 // per wave); the fixed cost (1.5 passes over W) was fitted to measured launches of 13 k and 32 k rows.
 struct SplitPlan {
     int m_tiles, units, mb, splits, waves;
+    int mb_last, splits_last;          // paired kernel only: a partial last wave split over more pairs per tile
     double cost;
 };
 
@@ -197,7 +201,7 @@ SplitPlan plan_split(int M, int V, int D, int workers, int tile_rows, int unit, 
     SplitPlan p;
     p.m_tiles = (M + tile_rows - 1) / tile_rows;
     p.units = (V + unit - 1) / unit;
-    p.mb = p.splits = p.waves = 0;
+    p.mb = p.splits = p.waves = p.mb_last = p.splits_last = 0;
     p.cost = 0.0;
     const double flops_per_sm = 1.0e13, hbm = 6.0e12;
     for (int waves = 1; waves <= p.m_tiles; ++waves) {
@@ -217,6 +221,47 @@ SplitPlan plan_split(int M, int V, int D, int workers, int tile_rows, int unit, 
     return p;
 }
 
+// Work split of the paired kernel: 256-row tiles, granules of 32 vocabulary entries, `pairs` pairs of SMs.  Every
+// full wave has mb tiles in flight, each swept by `splits` pairs (mb * splits <= pairs); what is left of the tiles
+// makes a last wave of mb_last tiles, each swept by splits_last = pairs / mb_last pairs, so that no pair sits out a
+// whole sweep because the tile count is not a multiple of mb.  The hidden states of a wave (mb tiles, re-read from L2
+// once per vocabulary tile) must stay L2-resident beside the weight stream, which bounds mb: measured at 32768 and
+// 103042 rows with budgets of 30 / 40 / 52 / 64 / 80 MB (6 / 4 / 3 / 3 / 2 pairs per tile): 1382 / 1386 / 1378 / 1381 /
+// 1346 and 1373 / 1391 / 1367 / 1362 / 1307 TFLOP/s under the power cap.  Cost as in plan_split.
+constexpr long long kMaxWaveHiddenBytes = 40ll << 20;
+
+SplitPlan plan_pair_split(int M, int V, int D, int pairs)
+{
+    SplitPlan p;
+    p.m_tiles = (M + 2 * kTileM - 1) / (2 * kTileM);
+    p.units = (V + kPairUnit - 1) / kPairUnit;
+    p.mb = p.splits = p.waves = p.mb_last = p.splits_last = 0;
+    p.cost = 0.0;
+    const double flops_per_sm = 1.0e13, hbm = 6.0e12;
+    const double t_unit = (double)kPairUnit * kTileM * 2.0 * D / flops_per_sm, t_hbm = 2.0 * V * (double)D / hbm;
+    for (int splits = 1; splits <= pairs && splits <= p.units; ++splits) {
+        int mb = pairs / splits;
+        if (mb > p.m_tiles) mb = p.m_tiles;
+        if ((long long)mb * 2 * kTileM * D * 2 > kMaxWaveHiddenBytes && mb > 1) continue;
+        const int full = p.m_tiles / mb, rest = p.m_tiles % mb;
+        int splits_last = 0;
+        if (rest > 0) {
+            splits_last = pairs / rest;
+            if (splits_last > p.units) splits_last = p.units;
+        }
+        const int waves = full + (rest > 0 ? 1 : 0);
+        const double t_full = (double)((p.units + splits - 1) / splits) * t_unit;
+        const double t_rest = rest > 0 ? (double)((p.units + splits_last - 1) / splits_last) * t_unit : 0.0;
+        const double cost = full * ((t_full > t_hbm ? t_full : t_hbm) + 1.5 * t_hbm) +
+                            (rest > 0 ? (t_rest > t_hbm ? t_rest : t_hbm) + 1.5 * t_hbm : 0.0);
+        if (p.waves == 0 || cost < p.cost * 0.999) {
+            p.cost = cost; p.waves = waves; p.mb = mb; p.splits = splits;
+            p.mb_last = rest; p.splits_last = splits_last;
+        }
+    }
+    return p;
+}
+
 }  // namespace
 
 pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool allow_swapped)
@@ -227,13 +272,12 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool al
     g.a_rows = tiles128 == 1 ? ((M + 7) / 8) * 8 : kTileM;
     SplitPlan p = plan_split(M, V, D, n_sm, kTileM, kUnit, kMaxConcurrentTiles);
     g.paired = 0;
-    if (tiles128 >= kPairMinTiles && M <= kPairMaxRows && n_sm >= 2) {
-        // The paired kernel works on 256-row tiles, granules of 32 vocabulary entries and pairs of SMs.  It
-        // feeds the tensor cores better (measured: +8 .. +29 % from 129 to 8192 rows); it loses where pairs
-        // and 256-row tiles divide the work less evenly, and in long launches the power cap, not the operand
-        // feed, sets the pace (16 k rows and more: the single-block kernel is 4 .. 6 % faster).
-        const SplitPlan pp = plan_split(M, V, D, n_sm / 2, 2 * kTileM, kPairUnit, kMaxConcurrentTiles / 2);
-        if (pp.waves > 0 && pp.cost <= 1.05 * p.cost) { p = pp; g.paired = 1; }
+    if (tiles128 >= kPairMinTiles && n_sm >= 2) {
+        // The paired kernel works on 256-row tiles, granules of 32 vocabulary entries and pairs of SMs: each SM
+        // pulls a third less through L2 per MMA cycle, which is what bounds the single-block kernel (and costs
+        // power: under the cap the paired kernel does the same work at a lower clock).
+        const SplitPlan pp = plan_pair_split(M, V, D, n_sm / 2);
+        if (pp.waves > 0) { p = pp; g.paired = 1; }
     }
     g.swapped = 0; g.n_pad = 0; g.stages = 0;
     if (allow_swapped && n_sm >= 2 && ((M > kStreamRows && M <= kSwapSmallMaxRows) || (M > kTileM && M <= kSwapRaggedMaxRows) ||
@@ -250,8 +294,11 @@ pvf_score_geometry pvf_score_geometry_for(int M, int V, int D, int n_sm, bool al
     }
     g.m_tiles = p.m_tiles; g.units = p.units;
     g.mb = p.mb; g.splits = p.splits; g.waves = p.waves;
-    g.ctas = g.mb * g.splits * ((g.paired || g.swapped) ? 2 : 1);
-    g.parts = g.splits * (g.swapped ? 2 : 1);
+    g.mb_last = g.paired ? p.mb_last : 0; g.splits_last = g.paired ? p.splits_last : 0;
+    int workers = g.mb * g.splits;
+    if (g.mb_last * g.splits_last > workers) workers = g.mb_last * g.splits_last;
+    g.ctas = workers * ((g.paired || g.swapped) ? 2 : 1);
+    g.parts = (g.splits_last > g.splits ? g.splits_last : g.splits) * (g.swapped ? 2 : 1);
     return g;
 }
 
@@ -283,8 +330,8 @@ int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, 
     const pvf_score_geometry g = pvf_score_geometry_for(M, V, D, ctx->n_sm);
     if ((size_t)M * g.parts * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
     *parts = g.parts;
-    return launch_projection(g, hidden, M, V, D, ctx->tm_w, ctx->partials, &ctx->words->status, (cudaStream_t)stream,
-                             ctx->ev_start, ctx->ev_stop);
+    return launch_projection(g, hidden, M, V, D, ctx->tm_w, ctx->partials, &ctx->words->status, &ctx->words->wave_arrivals,
+                             (cudaStream_t)stream, ctx->ev_start, ctx->ev_stop);
 }
 
 int pvf_score_init(pvf_ctx *ctx)
@@ -316,7 +363,8 @@ int pvf_score_plan(pvf_ctx *ctx, int32_t M, int32_t *ctas, int32_t *splits, int3
 }
 
 int pvf_score_plan_for_shape(int32_t vocab, int32_t hidden, int32_t n_sm, int32_t M, int32_t *ctas, int32_t *splits,
-                             int32_t *waves, int32_t *kernel, int32_t *row_tiles, int32_t *tiles_per_wave)
+                             int32_t *waves, int32_t *kernel, int32_t *row_tiles, int32_t *tiles_per_wave,
+                             int32_t *last_wave_tiles, int32_t *last_wave_splits)
 {
     if (vocab <= 0 || hidden <= 0 || n_sm <= 0 || M <= 0) return PVF_ERR_INVALID;
     const pvf_score_geometry g = pvf_score_geometry_for(M, vocab, hidden, n_sm);
@@ -326,6 +374,8 @@ int pvf_score_plan_for_shape(int32_t vocab, int32_t hidden, int32_t n_sm, int32_
     if (kernel) *kernel = g.streaming ? 0 : (g.swapped ? 3 : (g.paired ? 2 : 1));
     if (row_tiles) *row_tiles = g.m_tiles;
     if (tiles_per_wave) *tiles_per_wave = g.mb;
+    if (last_wave_tiles) *last_wave_tiles = g.mb_last;
+    if (last_wave_splits) *last_wave_splits = g.splits_last;
     return PVF_OK;
 }
 
@@ -429,7 +479,7 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     // The array keeps the previous call's contents.  The status word must start at zero; the partial
     // states need no clearing: the projection kernel writes every (row, range) entry the merge kernel reads.
     if (cudaMemsetAsync(status, 0, sizeof(int32_t), s) != cudaSuccess) return PVF_ERR_CUDA;
-    if ((rc = launch_projection(g, hidden, M, vocab, hidden_size, w_levels, partials, status, s, nullptr, nullptr)) != PVF_OK) return rc;
+    if ((rc = launch_projection(g, hidden, M, vocab, hidden_size, w_levels, partials, status, nullptr, s, nullptr, nullptr)) != PVF_OK) return rc;
     return launch_merge(partials, M, g.parts, vocab, plan_bitmap, tok, conf, ent, in_plan, s);
 }
 

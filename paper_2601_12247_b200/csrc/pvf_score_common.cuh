@@ -15,7 +15,6 @@ constexpr int kGeneralTileN = 256;         // 128-row GEMM kernel: vocabulary en
 constexpr int kGeneralPanels = 1;          //   64-element k-panels per pipeline stage
 constexpr int kGeneralStages = 4;          //   pipeline stages
 constexpr int kPairMinTiles = 2;           // 128-row tiles from which the paired (cta_group::2) kernel takes over
-constexpr int kPairMaxRows = 8192;         // rows up to which the paired kernel is considered
 constexpr int kSwapSmallMaxRows = 64;      // 33 .. this many rows take the swapped paired kernel
 constexpr int kSwapRaggedMaxRows = 192;    // and so do 129 .. this many rows (at most 256)
 constexpr int kSwapWideWarps = 3;          // epilogue warps per lane quadrant of the swapped paired kernel above 256 rows
@@ -77,12 +76,14 @@ struct ScoreArgs {
     int num_kb;          // ceil(D / 64)
     int units;           // ceil(V / 16)
     int m_tiles, mb, splits, waves;
+    int mb_last, splits_last;   // paired kernel: geometry of a partial last wave (mb_last = 0: every wave is full)
     int a_rows;          // rows per H box
     int n_pad, stages;   // swapped paired kernel: rows per row tile (MMA N), pipeline stages
     int w_once;          // 1: the launch reads every W tile exactly once (its L2 lines are marked evict-first)
     int parts;           // partial states per row (row stride of `partials`)
     float4 *partials;    // [M][parts]
     int32_t *status;
+    uint32_t *wave_sync; // paired kernel with several waves: {arrivals, done} counters of the wave boundaries, else nullptr
 };
 
 // ---------------------------------------------------------------------------------- PTX helpers
@@ -148,13 +149,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 
 // L2 eviction priority for the W tiles.  Where a launch reads W exactly once (one wave, one row tile in flight) the
 // tiles are marked evict-first: a gigabyte of weights then streams through L2 without pushing out what the small
-// kernels behind the projection need (their instructions, the partial states, the hidden states); where blocks share W
-// tiles through L2 (several row tiles in flight) the priority stays normal.
-__device__ __forceinline__ uint64_t w_l2_policy(int read_once)
+// kernels behind the projection need (their instructions, the partial states, the hidden states).  Where blocks share
+// W tiles through L2 (several row tiles in flight) the loads carry no hint at all: the hinted form of the instruction,
+// even with the normal priority, cost 3 % (paired kernel) to 11 % (128-row kernel) at 32768 rows.
+__device__ __forceinline__ uint64_t w_evict_first_policy()
 {
     uint64_t p;
-    if (read_once) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
     return p;
 }
 __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap *map, uint32_t bar, int x, int y, uint64_t policy)
@@ -345,9 +346,11 @@ __device__ __forceinline__ void fold16(RowState &st, const uint32_t (&raw)[16], 
 
 
 // One W tile of `tun` granules starting at granule tu0, columns x .. x+63, into b_dst.
+template <bool kReadOnce>
 __device__ __forceinline__ void load_w_tile(uint32_t b_dst, const WMaps &maps, uint32_t full, int x, int tu0, int tun, uint64_t policy)
 {
-    tma_load_2d_hint(b_dst, &maps.size[tun - 1], full, x, tu0 * kUnit, policy);
+    if (kReadOnce) tma_load_2d_hint(b_dst, &maps.size[tun - 1], full, x, tu0 * kUnit, policy);
+    else tma_load_2d(b_dst, &maps.size[tun - 1], full, x, tu0 * kUnit);
 }
 
 }  // namespace

@@ -6,6 +6,48 @@
 namespace {
 
 // ---------------------------------------------------------------------------------- GEMM kernel
+// The TMA producer's loop (one thread).  kReadOnce: W is read exactly once by the launch (evict-first hint).
+template <class Cfg, bool kReadOnce>
+__device__ __forceinline__ void gemm_produce(const ScoreArgs &args, const CUtensorMap &tm_h, const WMaps &tm_w, SharedControl *ctl,
+                                             const TileSplit &split, uint32_t tiles_addr, int mt_local, int k_steps)
+{
+    constexpr int kStages = Cfg::kStages;
+    constexpr int kPanels = Cfg::kPanels;
+    const int n_tiles = split.n_tiles;
+    int stage = 0;
+    uint32_t phase = 0;
+    ArmedStages armed;
+    const uint64_t w_policy = kReadOnce ? w_evict_first_policy() : 0ull;
+    bool alive = true;
+    for (int w = 0; w < args.waves && alive; ++w) {
+        const int m_tile = w * args.mb + mt_local;
+        if (m_tile >= args.m_tiles) continue;
+        for (int tile = 0; tile < n_tiles && alive; ++tile) {
+            int tu0, tun;                                              // first granule, granules of this tile
+            split.tile(tile, &tu0, &tun);
+            const uint32_t panel_bytes = (uint32_t)args.a_rows * kRowBytes + (uint32_t)tun * kUnitBytes;
+            for (int step = 0; step < k_steps; ++step) {
+                const int kb0 = step * kPanels;
+                const int np = min(kPanels, args.num_kb - kb0);
+                if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                const uint32_t full = smem_u32(&ctl->full[stage]);
+                const uint32_t a_base = tiles_addr + stage * Cfg::kStageBytes;
+                const uint32_t b_base = a_base + kPanels * Cfg::kAPanelBytes;
+                mbar_arrive_expect_tx(full, panel_bytes * (uint32_t)np);
+                armed.note(stage, phase);
+                for (int p = 0; p < np; ++p) {
+                    const int x = (kb0 + p) * kBlockK;
+                    tma_load_2d(a_base + p * Cfg::kAPanelBytes, &tm_h, full, x, m_tile * kTileM);
+                    load_w_tile<kReadOnce>(b_base + p * Cfg::kBPanelBytes, tm_w, full, x, tu0, tun, w_policy);
+                }
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+    // Abort: let every copy this thread started land before the block's memory is released.
+    if (!alive) drain_armed_stages(ctl, armed, kStages);
+}
+
 template <class Cfg>
 __global__ void __launch_bounds__(kThreads, 1)
 pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ WMaps tm_w, const ScoreArgs args)
@@ -53,38 +95,8 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            ArmedStages armed;
-            const uint64_t w_policy = w_l2_policy(args.w_once);
-            bool alive = true;
-            for (int w = 0; w < args.waves && alive; ++w) {
-                const int m_tile = w * args.mb + mt_local;
-                if (m_tile >= args.m_tiles) continue;
-                for (int tile = 0; tile < n_tiles && alive; ++tile) {
-                    int tu0, tun;                                              // first granule, granules of this tile
-                    split.tile(tile, &tu0, &tun);
-                    const uint32_t panel_bytes = (uint32_t)args.a_rows * kRowBytes + (uint32_t)tun * kUnitBytes;
-                    for (int step = 0; step < k_steps; ++step) {
-                        const int kb0 = step * kPanels;
-                        const int np = min(kPanels, args.num_kb - kb0);
-                        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
-                        const uint32_t full = smem_u32(&ctl->full[stage]);
-                        const uint32_t a_base = tiles_addr + stage * Cfg::kStageBytes;
-                        const uint32_t b_base = a_base + kPanels * Cfg::kAPanelBytes;
-                        mbar_arrive_expect_tx(full, panel_bytes * (uint32_t)np);
-                        armed.note(stage, phase);
-                        for (int p = 0; p < np; ++p) {
-                            const int x = (kb0 + p) * kBlockK;
-                            tma_load_2d(a_base + p * Cfg::kAPanelBytes, &tm_h, full, x, m_tile * kTileM);
-                            load_w_tile(b_base + p * Cfg::kBPanelBytes, tm_w, full, x, tu0, tun, w_policy);
-                        }
-                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
-                    }
-                }
-            }
-            // Abort: let every copy this thread started land before the block's memory is released.
-            if (!alive) drain_armed_stages(ctl, armed, kStages);
+            if (args.w_once) gemm_produce<Cfg, true>(args, tm_h, tm_w, ctl, split, tiles_addr, mt_local, k_steps);
+            else gemm_produce<Cfg, false>(args, tm_h, tm_w, ctl, split, tiles_addr, mt_local, k_steps);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer

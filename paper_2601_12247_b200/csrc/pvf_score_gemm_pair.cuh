@@ -86,6 +86,95 @@ __device__ __forceinline__ uint32_t instr_desc_bf16_m256(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 }
 
+// Work of pair `pair` in wave w: its 256-row tile, its vocabulary range (granules of 32) and the index q of that
+// range among the tile's.  Every wave but a partial last one has args.mb tiles in flight, each swept by args.splits
+// pairs; a partial last wave has args.mb_last tiles and args.splits_last (more) pairs per tile, so that the pairs
+// are all busy there too.  False: the pair has nothing to do in this wave.
+__device__ __forceinline__ bool pair_wave_work(const ScoreArgs &args, int pair, int w, int *s_tile, int *q, int *u0, int *u1)
+{
+    const bool last = args.mb_last > 0 && w == args.waves - 1;
+    const int mb = last ? args.mb_last : args.mb, splits = last ? args.splits_last : args.splits;
+    *q = pair / mb;
+    *s_tile = w * args.mb + pair % mb;
+    if (*q >= splits || *s_tile >= args.m_tiles) return false;
+    split_range(args.units, splits, *q, u0, u1);
+    return true;
+}
+
+// Wave boundary.  The blocks that sweep one vocabulary range for different row tiles stream the same W tiles, and
+// W crosses HBM once per wave only while they stay close together (what one block fetched, the others find in L2).
+// Over several waves they drift apart -- measured: 1356 TFLOP/s at 2 waves, 1150 at 17 -- so every block's producer
+// thread waits at the start of each wave until all blocks of the grid have got there (the launch is cooperative: all
+// blocks are resident).  The wait is bounded like every other.
+__device__ __forceinline__ bool wave_boundary(uint32_t *arrivals, unsigned target, SharedControl *ctl, int32_t *status)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(arrivals) : "memory");
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
+        unsigned seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(arrivals) : "memory");
+        if (seen >= target) return true;
+        if (ctl->abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) {
+            ctl->abort_flag = 1;
+            atomicExch(status, (int32_t)PVF_ERR_TIMEOUT);
+            return false;
+        }
+        __nanosleep(256);
+    }
+}
+
+// The TMA producer's loop (one thread per block).  kReadOnce: W is read exactly once by the launch (evict-first hint).
+template <bool kReadOnce>
+__device__ __forceinline__ void pair_produce(const ScoreArgs &args, const CUtensorMap &tm_h, const WMaps &tm_w, SharedControl *ctl,
+                                             uint32_t tiles_addr, int pair, uint32_t rank, int k_steps)
+{
+    int stage = 0;
+    uint32_t phase = 0;
+    ArmedStages armed;                                                       // even block: it arms full[]
+    const uint64_t w_policy = kReadOnce ? w_evict_first_policy() : 0ull;
+    bool alive = true;
+    for (int w = 0; w < args.waves && alive; ++w) {
+        if (w > 0 && args.wave_sync && !wave_boundary(args.wave_sync, (unsigned)w * gridDim.x, ctl, args.status)) { alive = false; break; }
+        int s_tile, q, u0, u1;
+        if (!pair_wave_work(args, pair, w, &s_tile, &q, &u0, &u1)) continue;
+        const TileSplit split(u0, u1, kPairUnitsPerTile);
+        const int n_tiles = split.n_tiles;
+        const int row0 = s_tile * 2 * kTileM + (int)rank * kTileM;          // this block's rows
+        for (int tile = 0; tile < n_tiles && alive; ++tile) {
+            int tu0, tun;
+            split.tile(tile, &tu0, &tun);
+            const uint32_t bytes = 2u * ((uint32_t)kPairABytes + (uint32_t)tun * kUnitBytes);   // both blocks
+            const int w_row = tu0 * kPairUnit + (int)rank * tun * kUnit;                        // this block's half
+            for (int step = 0; step < k_steps; ++step) {
+                if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                const uint32_t full = smem_u32(&ctl->full[stage]);
+                const uint32_t a_dst = tiles_addr + stage * kPairStageBytes;
+                if (rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
+                tma_load_2d_pair(a_dst, &tm_h, full, step * kBlockK, row0);
+                if (kReadOnce) tma_load_2d_pair_hint(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
+                else tma_load_2d_pair(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
+                if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+    }
+    if (alive && args.wave_sync && args.waves > 1 && atomicAdd(args.wave_sync + 1, 1u) == gridDim.x - 1) {
+        args.wave_sync[0] = 0;                                               // every block is past its last boundary:
+        args.wave_sync[1] = 0;                                               // rearm the counters for the next launch
+    }
+    if (!alive) {
+        // Abort: the copies in flight land before the pair leaves.  The even block's full[] barriers count
+        // both blocks' bytes, so it waits (bounded) on every stage it armed; the odd block has no barrier
+        // of its own to wait on and gives its copies a fixed time (the closing cluster barrier holds both
+        // blocks until the slower one is through).
+        if (rank == 0) drain_armed_stages(ctl, armed, kPairStages);
+        else {
+            const unsigned long long t0 = global_timer_ns();
+            while (global_timer_ns() - t0 < 200000ull) {}
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_constant__ WMaps tm_w, const ScoreArgs args)
 {
@@ -99,12 +188,6 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     const int lane = threadIdx.x & 31;
     const uint32_t rank = cluster_cta_rank();                            // 0: even block (issues the MMAs), 1: its peer
     const int pair = blockIdx.x >> 1;
-    const int st_local = pair % args.mb;                                 // 256-row tile of the wave
-    const int q = pair / args.mb;                                        // vocabulary range
-    int u0, u1;
-    split_range(args.units, args.splits, q, &u0, &u1);                   // granules of 32 entries
-    const TileSplit split(u0, u1, kPairUnitsPerTile);
-    const int n_tiles = split.n_tiles;
     const int k_steps = args.num_kb;
 
     if (threadIdx.x == 0) init_pipeline_barriers(ctl, kPairStages, 1, 2 * kEpilogueThreads);
@@ -127,42 +210,8 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (one per block)
         if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            ArmedStages armed;
-            const uint64_t w_policy = w_l2_policy(args.w_once);
-            bool alive = true;
-            for (int w = 0; w < args.waves && alive; ++w) {
-                const int s_tile = w * args.mb + st_local;
-                if (s_tile >= args.m_tiles) continue;
-                const int row0 = s_tile * 2 * kTileM + (int)rank * kTileM;          // this block's rows
-                for (int tile = 0; tile < n_tiles && alive; ++tile) {
-                    int tu0, tun;
-                    split.tile(tile, &tu0, &tun);
-                    const uint32_t bytes = 2u * ((uint32_t)kPairABytes + (uint32_t)tun * kUnitBytes);   // both blocks
-                    const int w_row = tu0 * kPairUnit + (int)rank * tun * kUnit;                        // this block's half
-                    for (int step = 0; step < k_steps; ++step) {
-                        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
-                        const uint32_t full = smem_u32(&ctl->full[stage]);
-                        const uint32_t a_dst = tiles_addr + stage * kPairStageBytes;
-                        if (rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
-                        tma_load_2d_pair(a_dst, &tm_h, full, step * kBlockK, row0);
-                        tma_load_2d_pair_hint(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
-                        if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
-                    }
-                }
-            }
-            if (!alive) {
-                // Abort: the copies in flight land before the pair leaves.  The even block's full[] barriers count
-                // both blocks' bytes, so it waits (bounded) on every stage it armed; the odd block has no barrier
-                // of its own to wait on and gives its copies a fixed time (the closing cluster barrier holds both
-                // blocks until the slower one is through).
-                if (rank == 0) drain_armed_stages(ctl, armed, kPairStages);
-                else {
-                    const unsigned long long t0 = global_timer_ns();
-                    while (global_timer_ns() - t0 < 200000ull) {}
-                }
-            }
+            if (args.w_once) pair_produce<true>(args, tm_h, tm_w, ctl, tiles_addr, pair, rank, k_steps);
+            else pair_produce<false>(args, tm_h, tm_w, ctl, tiles_addr, pair, rank, k_steps);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even block only)
@@ -172,8 +221,10 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             uint32_t tile_count = 0;
             bool alive = true;
             for (int w = 0; w < args.waves && alive; ++w) {
-                const int s_tile = w * args.mb + st_local;
-                if (s_tile >= args.m_tiles) continue;
+                int s_tile, q, u0, u1;
+                if (!pair_wave_work(args, pair, w, &s_tile, &q, &u0, &u1)) continue;
+                const TileSplit split(u0, u1, kPairUnitsPerTile);
+                const int n_tiles = split.n_tiles;
                 for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
                     int tu0, tun;
                     split.tile(tile, &tu0, &tun);
@@ -213,8 +264,10 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
         uint32_t tile_count = 0;
         bool alive = true;
         for (int w = 0; w < args.waves && alive; ++w) {
-            const int s_tile = w * args.mb + st_local;
-            if (s_tile >= args.m_tiles) continue;
+            int s_tile, q, u0, u1;
+            if (!pair_wave_work(args, pair, w, &s_tile, &q, &u0, &u1)) continue;
+            const TileSplit split(u0, u1, kPairUnitsPerTile);
+            const int n_tiles = split.n_tiles;
             const int row_base = s_tile * 2 * kTileM + (int)rank * kTileM;
             const int row = row_base + row_in_tile;
             const bool warp_has_rows = row_base + quad * 32 < args.M;
@@ -242,8 +295,14 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
                 tc_fence_before_sync();
                 mbar_arrive_even_block(smem_u32(&ctl->acc_empty[buf]));
             }
-            if (alive && row < args.M)
-                args.partials[(size_t)row * args.splits + q] = make_float4(st.m, st.s, st.t, __int_as_float(st.arg));
+            if (alive && row < args.M) {
+                float4 *row_parts = args.partials + (size_t)row * args.parts;
+                row_parts[q] = make_float4(st.m, st.s, st.t, __int_as_float(st.arg));
+                // a row's slots beyond its wave's ranges (the other kind of wave has more) hold empty states
+                const int splits = (args.mb_last > 0 && w == args.waves - 1) ? args.splits_last : args.splits;
+                if (q == 0)
+                    for (int e = splits; e < args.parts; ++e) row_parts[e] = make_float4(-INFINITY, 0.f, 0.f, __int_as_float(kNoArg));
+            }
         }
     }
 

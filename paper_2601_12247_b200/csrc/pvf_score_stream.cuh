@@ -96,7 +96,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
             int stage = 0;
             uint32_t phase = 0;
             ArmedStages armed;
-            const uint64_t w_policy = w_l2_policy(args.w_once);
+            const uint64_t w_policy = w_evict_first_policy();         // one wave, one row tile: W is read once
             bool alive = true;
             for (int tile = 0; tile < n_tiles && alive; ++tile) {
                 int tu0, tun;
@@ -109,7 +109,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
                     mbar_arrive_expect_tx(full, bytes);
                     armed.note(stage, phase);
                     tma_load_2d(h_dst, &tm_h, full, step * kBlockK, 0);
-                    load_w_tile(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, w_policy);
+                    load_w_tile<true>(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, w_policy);
                     if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
                 }
             }

@@ -71,7 +71,7 @@ inline int swap_stages(int n_pad)
 // two threads set the pace of the kernel, and a run-time choice inside their loops costs more than it looks.
 struct SwapLoopArgs {
     uint32_t tiles_addr, stage_bytes, h0_bytes, h1_bytes, tmem_base;
-    int n0, n1, n_stages, n_tiles, k_steps, n_bufs, w_once;
+    int n0, n1, n_stages, n_tiles, k_steps, n_bufs;
     uint32_t rank;
 };
 
@@ -84,7 +84,7 @@ __device__ __forceinline__ void swap_produce(const SwapLoopArgs &a, const TileSp
     uint32_t phase = 0;
     bool alive = true;
     ArmedStages armed;
-    const uint64_t w_policy = w_l2_policy(a.w_once);
+    const uint64_t w_policy = w_evict_first_policy();            // one wave, one row tile: W is read once
     const int row0 = (int)a.rank * (a.n0 / 2);                                      // this block's half of each group's rows
     const int row1 = a.n0 + (int)a.rank * (a.n1 / 2);
     for (int tile = 0; tile < a.n_tiles && alive; ++tile) {
@@ -214,7 +214,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     SwapLoopArgs la;
     la.tiles_addr = tiles_addr; la.stage_bytes = stage_bytes; la.h0_bytes = h0_bytes; la.h1_bytes = h1_bytes;
     la.tmem_base = tmem_base; la.n0 = n0; la.n1 = n1; la.n_stages = n_stages; la.n_tiles = n_tiles; la.k_steps = k_steps;
-    la.n_bufs = n_bufs; la.rank = rank; la.w_once = args.w_once;
+    la.n_bufs = n_bufs; la.rank = rank;
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (one per block)
         if (lane == 0) {

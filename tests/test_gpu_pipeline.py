@@ -387,8 +387,8 @@ def torch_fp64_reference(w_head, h_dev, chunk=1024):
 
 
 def test_config3_verification_pass_sampled():
-    # Config 3's verification pass at its stated size: the 64 sequences' (1 + K_t) * |R_b| rows (about 10^5, several
-    # passes over W of the 128-row kernel) scored in the geometry the benchmark times.  Sampled rows against the
+    # Config 3's verification pass at its stated size: the 64 sequences' (1 + K_t) * |R_b| rows (about 10^5, eleven
+    # passes over W of the paired kernel, the last one a partial wave) scored in the geometry the benchmark times.  Sampled rows against the
     # oracle one by one, every row against the torch fp64 reference that is pinned to the oracle on that sample, and
     # pvf_verify on the GPU's own fp32 numbers against the oracle's rule fed the same numbers.
     w_bits = synth.make_w(1001, synth.LLADA_VOCAB, synth.LLADA_HIDDEN)
@@ -418,7 +418,8 @@ def test_config3_verification_pass_sampled():
     Mv = int(v.hv_bits.shape[0])
     assert np.array_equal(v.v_off, osel["v_off"]) and Mv > 65536
     geo = ctx.score_plan(Mv)
-    assert geo["waves"] >= 8 and ctx.score_kernel_name(Mv) == "pvf_score_gemm_kernel"
+    assert geo["waves"] >= 8 and ctx.score_kernel_name(Mv) == "pvf_score_gemm_pair_kernel"
+    full = binding.score_plan_for_shape(st.vocab, st.hidden, torch.cuda.get_device_properties(0).multi_processor_count, Mv)
     hv = upload_bits(v.hv_bits)
     scv = ctx.score(hv)
     ver = ctx.verify(prm, seg, pos, sel, sc["tok"], scv["tok"], scv["conf"], cm["commit"])
@@ -428,10 +429,11 @@ def test_config3_verification_pass_sampled():
     check_score_properties(g_scv, st.vocab, plan)
     # sampled rows: first and last row, both sides of a 128-row tile edge, of a wave edge (rows per pass over W) and
     # of sequence boundaries of the [b][c][r] layout
-    rows_per_wave = 128 * ((Mv + 127) // 128 + geo["waves"] - 1) // geo["waves"]
-    rows_per_wave = min(rows_per_wave, Mv - 1)
-    sample = np.unique(np.clip(np.array([0, 127, 128, rows_per_wave - 1, rows_per_wave, int(v.v_off[1]) - 1, int(v.v_off[1]),
-                                         int(v.v_off[32]), Mv // 2, Mv - 129, Mv - 128, Mv - 1]), 0, Mv - 1))
+    rows_per_wave = min(256 * full["tiles_per_wave"], Mv - 1)
+    last_wave = rows_per_wave * (full["waves"] - 1)                   # first row of the last wave (split over more pairs)
+    sample = np.unique(np.clip(np.array([0, 127, 128, 255, 256, rows_per_wave - 1, rows_per_wave, int(v.v_off[1]) - 1,
+                                         int(v.v_off[1]), int(v.v_off[32]), Mv // 2, last_wave - 1, last_wave, Mv - 129,
+                                         Mv - 128, Mv - 1]), 0, Mv - 1))
     want = oscore.score(w_bits, v.hv_bits[sample], plan)
     check_score(g_scv, want, st.vocab, plan, rows=sample)
     ref_conf, ref_ent, ref_tok, ref_gap = torch_fp64_reference(ctx.w_head, hv)
