@@ -342,6 +342,7 @@ def run_workload(name, synth, binding, dev, world, rank, local_rank, peaks, step
     for _ in range(max(warmup, 3)):
         step(h, hv)
     barrier()
+    ctx.score_clock(0); ctx.score_clock(1)             # clear the device-side clock sums of the projection launches
     sampler = ClockSampler(gpu_id_of(dev, local_rank))
     sampler.start()
     launches, n_steps_run = 0, 0
@@ -362,6 +363,9 @@ def run_workload(name, synth, binding, dev, world, rank, local_rank, peaks, step
         if enough or len(block_ms) >= MAX_REPEATS:
             break
     clocks = sampler.stop()
+    device_clock = {M: ctx.score_clock(0)}             # SM clock and cycles of the projection launches, measured by the kernels
+    if Mv:
+        device_clock[Mv] = ctx.score_clock(1)
     ctx.set_score_events(None, None)
     median_block = int(np.argsort(block_ms)[len(block_ms) // 2])
     ms = float(block_ms[median_block])
@@ -372,6 +376,12 @@ def run_workload(name, synth, binding, dev, world, rank, local_rank, peaks, step
     used = [(a, b, r) for a, b, r, blk in ev_pairs if event_every > 1 or blk == median_block]
     roof = roofline_of(used, ctx, V, D, peaks, clocks.get("sm_mhz"), event_every)
     roof["launches_timed_in"] = "the median block" if event_every == 1 else "all blocks"
+    # the kernels' own measurement over every launch of the timed region: run time and SM cycles of their first block
+    for item in roof["per_row_count"]:
+        c = device_clock.get(item["rows"])
+        if c and c["launches"]:
+            item.update(device_sm_mhz=c["sm_mhz"], device_kernel_us=1e3 * c["ms"], device_sm_cycles=c["sm_cycles"],
+                        device_launches=c["launches"])
 
     # ---------------- the same step captured once in a CUDA graph and replayed (no per-launch host work, no events
     # between the kernels): reported beside the main number

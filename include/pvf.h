@@ -156,6 +156,17 @@ const char *pvf_score_kernel_name(pvf_ctx *ctx, int32_t M);
 int pvf_set_score_events(pvf_ctx *ctx, void *start, void *stop);
 
 /*
+ * SM clock of the projection launches, measured on the device.  Every projection kernel's first block adds its own
+ * run time (nanoseconds) and SM cycle count to sums kept in the workspace; this call synchronises the device, returns
+ * the averages since the last call and clears the sums.  pass 0 = pvf_score and pvf_draft_step, 1 = pvf_verify_step.
+ *   ms        mean run time of the first block (close to the kernel's duration)       (may be NULL)
+ *   sm_mhz    cycles / time: the clock the launches really ran at under the power cap  (may be NULL)
+ *   launches  launches counted                                                          (may be NULL)
+ * ms * sm_mhz * 1000 = SM cycles per launch: what separates a kernel's efficiency from the clock it was given.
+ */
+int pvf_score_clock(pvf_ctx *ctx, int32_t pass, double *ms, double *sm_mhz, int64_t *launches);
+
+/*
  * pvf_score -- the vocabulary pass of one forward (Section 2 "confidence-based parallel decoding";
  * Section 3, definitions of y^_t^i, p_t^i and H_i; Section 4.1, "y^ in P^plan").
  *

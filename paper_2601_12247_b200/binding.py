@@ -82,6 +82,8 @@ def load() -> ctypes.CDLL:
         lib.pvf_score_plan_for_shape.argtypes = [i32] * 4 + [ctypes.POINTER(i32)] * 8
         lib.pvf_score_plan_for_shape.restype = ctypes.c_int
         lib.pvf_score_kernel_name.argtypes = [vp, i32]; lib.pvf_score_kernel_name.restype = ctypes.c_char_p
+        lib.pvf_score_clock.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_int64)]
+        lib.pvf_score_clock.restype = ctypes.c_int
         lib.pvf_score.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]; lib.pvf_score.restype = ctypes.c_int
         lib.pvf_commit.argtypes = [vp, pp, i32, i32] + [vp] * 8 + [i32, vp]; lib.pvf_commit.restype = ctypes.c_int
         lib.pvf_select_drafts.argtypes = [vp, pp, i32, i32] + [vp] * 13 + [vp]; lib.pvf_select_drafts.restype = ctypes.c_int
@@ -208,6 +210,13 @@ class Context:
         v = [ctypes.c_int32() for _ in range(4)]
         _check(self.lib.pvf_score_plan(self.handle, int(M), *[ctypes.byref(x) for x in v]), "pvf_score_plan")
         return dict(ctas=v[0].value, splits=v[1].value, waves=v[2].value, launches=v[3].value)
+
+    def score_clock(self, which: int) -> Dict[str, float]:
+        """pvf_score_clock: mean run time, SM clock and count of the projection launches since the last call
+        (which = 0: pvf_score / draft pass, 1: verification pass); synchronises the device and clears the sums."""
+        ms, mhz, n = ctypes.c_double(), ctypes.c_double(), ctypes.c_int64()
+        _check(self.lib.pvf_score_clock(self.handle, int(which), ctypes.byref(ms), ctypes.byref(mhz), ctypes.byref(n)), "pvf_score_clock")
+        return dict(ms=ms.value, sm_mhz=mhz.value, launches=int(n.value), sm_cycles=ms.value * mhz.value * 1e3)
 
     def score_kernel_name(self, M: int) -> str:
         name = self.lib.pvf_score_kernel_name(self.handle, int(M))

@@ -18,7 +18,12 @@ struct pvf_device_words {
     uint32_t working_ticket; // the same for pvf_working_set
     uint32_t wave_arrivals; // paired projection kernel: blocks that have reached a wave boundary (all waves of a launch)
     uint32_t wave_done;     //    blocks that are past their last wave boundary; the last one clears both
-    uint32_t pad[59];
+    uint32_t pad0[3];
+    // SM clock of the projection launches, measured on the device (pvf_score_clock): per slot (0: pvf_score and the
+    // draft pass, 1: the verification pass) the sums over launches of block 0's wall time (ns, %globaltimer) and of its
+    // SM cycles (clock64), and the number of launches.
+    unsigned long long clock_acc[2][3];
+    uint32_t pad[44];
 };
 
 struct pvf_ctx {
@@ -70,7 +75,7 @@ size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm);
 int pvf_score_init(pvf_ctx *ctx);   // tensor maps of W, kernel attributes
 // The projection half of pvf_score alone: launches the kernel that leaves `*parts` partial softmax states per row in
 // ctx->partials (row stride *parts); the caller's next kernel on the stream merges them (pvf_merge_rows).
-int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, void *stream);
+int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, int clock_slot, void *stream);
 
 // Programmatic dependent launch.  Every kernel of the library is launched with pvf_launch and runs
 //     <set-up that touches no global memory>; pvf_launch_dependents(); pvf_grid_dependency_wait();
@@ -101,24 +106,22 @@ static inline cudaError_t pvf_launch(void (*kernel)(KArgs...), dim3 grid, dim3 b
 // The same for a kernel whose blocks form clusters of two along x (grid.x even).
 template <typename... KArgs, typename... Args>
 static inline cudaError_t pvf_launch_cluster2(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
-                                              cudaStream_t stream, bool cooperative, Args... args)
+                                              cudaStream_t stream, Args... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[3];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
-    attr[2].id = cudaLaunchAttributeCooperative;       // the launch fails unless every block can be resident at once
-    attr[2].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = cooperative ? 3 : 2;
+    cfg.numAttrs = 2;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 #endif

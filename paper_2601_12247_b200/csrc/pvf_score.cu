@@ -124,8 +124,8 @@ int raise_shared_memory_limits()
 
 // Launches the projection kernel (shape chosen by the geometry) on `s`: it leaves g.parts partial states per row.
 int launch_projection(const pvf_score_geometry &g, const void *hidden, int M, int V, int D, const CUtensorMap *w_levels,
-                      float4 *partials, int32_t *status, uint32_t *wave_sync, cudaStream_t s, cudaEvent_t ev_start,
-                      cudaEvent_t ev_stop)
+                      float4 *partials, int32_t *status, uint32_t *wave_sync, unsigned long long *clock_acc, cudaStream_t s,
+                      cudaEvent_t ev_start, cudaEvent_t ev_stop)
 {
     CUtensorMap tm_h;
     int rc = make_tensor_map(&tm_h, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)g.a_rows);
@@ -145,6 +145,7 @@ int launch_projection(const pvf_score_geometry &g, const void *hidden, int M, in
     a.partials = partials;
     a.status = status;
     a.wave_sync = (g.paired && g.waves > 1) ? wave_sync : nullptr;
+    a.clock_acc = clock_acc;
     const bool timed = ev_start && ev_stop;
     if (timed && cudaEventRecord(ev_start, s) != cudaSuccess) return PVF_ERR_CUDA;
     cudaError_t e;
@@ -153,10 +154,10 @@ int launch_projection(const pvf_score_geometry &g, const void *hidden, int M, in
         if (g.n_pad > kSwapGroupCols &&
             (rc = make_tensor_map(&tm_h1, hidden, (uint64_t)M, (uint64_t)D, (uint32_t)((g.n_pad - kSwapGroupCols) / 2))) != PVF_OK)
             return rc;
-        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(64 + 128 * swap_warps_per_quad(g.n_pad)), kSwapSmemBytes, s, false, tm_h, tm_h1, maps, a);
+        e = pvf_launch_cluster2(pvf_score_swap_pair_kernel, dim3(g.ctas), dim3(64 + 128 * swap_warps_per_quad(g.n_pad)), kSwapSmemBytes, s, tm_h, tm_h1, maps, a);
     }
     else if (g.paired)
-        e = pvf_launch_cluster2(pvf_score_gemm_pair_kernel, dim3(g.ctas), dim3(kThreads), kPairSmemBytes, s, a.wave_sync != nullptr, tm_h, maps, a);
+        e = pvf_launch_cluster2(pvf_score_gemm_pair_kernel, dim3(g.ctas), dim3(kThreads), kPairSmemBytes, s, tm_h, maps, a);
     else if (g.streaming)
         e = pvf_launch(pvf_score_stream_kernel, dim3(g.ctas), dim3(kStreamThreads), kStreamSmemBytes, s, tm_h, maps, a);
     else
@@ -322,7 +323,7 @@ size_t pvf_score_partials_bytes(const pvf_shape *shape, int n_sm)
     return worst;
 }
 
-int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, void *stream)
+int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, int clock_slot, void *stream)
 {
     if (!ctx || !parts || M <= 0 || M > ctx->shape.max_rows || !hidden) return PVF_ERR_INVALID;
     if (((uintptr_t)hidden & 15) != 0) return PVF_ERR_ALIGN;
@@ -331,7 +332,7 @@ int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, 
     if ((size_t)M * g.parts * sizeof(float4) > ctx->partials_bytes) return PVF_ERR_WORKSPACE;
     *parts = g.parts;
     return launch_projection(g, hidden, M, V, D, ctx->tm_w, ctx->partials, &ctx->words->status, &ctx->words->wave_arrivals,
-                             (cudaStream_t)stream, ctx->ev_start, ctx->ev_stop);
+                             ctx->words->clock_acc[clock_slot ? 1 : 0], (cudaStream_t)stream, ctx->ev_start, ctx->ev_stop);
 }
 
 int pvf_score_init(pvf_ctx *ctx)
@@ -348,6 +349,20 @@ int pvf_set_score_events(pvf_ctx *ctx, void *start, void *stop)
     if (!ctx || ((start == nullptr) != (stop == nullptr))) return PVF_ERR_INVALID;
     ctx->ev_start = (cudaEvent_t)start;
     ctx->ev_stop = (cudaEvent_t)stop;
+    return PVF_OK;
+}
+
+int pvf_score_clock(pvf_ctx *ctx, int32_t pass, double *ms, double *sm_mhz, int64_t *launches)
+{
+    if (!ctx || pass < 0 || pass > 1) return PVF_ERR_INVALID;
+    unsigned long long acc[3] = {0, 0, 0};
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpy(acc, ctx->words->clock_acc[pass], sizeof acc, cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemset(ctx->words->clock_acc[pass], 0, sizeof acc) != cudaSuccess)
+        return PVF_ERR_CUDA;
+    if (ms) *ms = acc[2] ? (double)acc[0] * 1e-6 / (double)acc[2] : 0.0;
+    if (sm_mhz) *sm_mhz = acc[0] ? (double)acc[1] * 1e3 / (double)acc[0] : 0.0;
+    if (launches) *launches = (int64_t)acc[2];
     return PVF_OK;
 }
 
@@ -394,7 +409,7 @@ int pvf_score(pvf_ctx *ctx, const void *hidden, int32_t M,
     if (M == 0) return PVF_OK;
     if (!hidden || !tok || !conf) return PVF_ERR_INVALID;
     int parts = 0;
-    const int rc = pvf_score_partials(ctx, hidden, M, &parts, stream);
+    const int rc = pvf_score_partials(ctx, hidden, M, &parts, 0, stream);
     if (rc != PVF_OK) return rc;
     return launch_merge(ctx->partials, M, parts, ctx->shape.vocab, ctx->plan_bitmap, tok, conf, ent, in_plan, (cudaStream_t)stream);
 }
@@ -479,7 +494,7 @@ int pvf_score_static(const void *w_head, int32_t vocab, int32_t hidden_size, con
     // The array keeps the previous call's contents.  The status word must start at zero; the partial
     // states need no clearing: the projection kernel writes every (row, range) entry the merge kernel reads.
     if (cudaMemsetAsync(status, 0, sizeof(int32_t), s) != cudaSuccess) return PVF_ERR_CUDA;
-    if ((rc = launch_projection(g, hidden, M, vocab, hidden_size, w_levels, partials, status, nullptr, s, nullptr, nullptr)) != PVF_OK) return rc;
+    if ((rc = launch_projection(g, hidden, M, vocab, hidden_size, w_levels, partials, status, nullptr, nullptr, s, nullptr, nullptr)) != PVF_OK) return rc;
     return launch_merge(partials, M, g.parts, vocab, plan_bitmap, tok, conf, ent, in_plan, s);
 }
 

@@ -84,6 +84,7 @@ struct ScoreArgs {
     float4 *partials;    // [M][parts]
     int32_t *status;
     uint32_t *wave_sync; // paired kernel with several waves: {arrivals, done} counters of the wave boundaries, else nullptr
+    unsigned long long *clock_acc;   // {ns, cycles, launches} sums of block 0's run (see LaunchClock), or nullptr
 };
 
 // ---------------------------------------------------------------------------------- PTX helpers
@@ -117,6 +118,25 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+
+// Block 0 measures its own run in wall time (%globaltimer) and in SM cycles (clock64) and adds both to the context's
+// sums: cycles / time is the SM clock the launch really ran at (the power cap moves it from launch to launch), and the
+// cycle count is what separates a kernel's efficiency from the clock it was given.
+struct LaunchClock {
+    unsigned long long t0, c0;
+    __device__ __forceinline__ void begin()
+    {
+        if (blockIdx.x == 0 && threadIdx.x == 0) { t0 = global_timer_ns(); c0 = (unsigned long long)clock64(); }
+    }
+    __device__ __forceinline__ void end(unsigned long long *acc) const
+    {
+        if (blockIdx.x == 0 && threadIdx.x == 0 && acc) {
+            atomicAdd(acc, global_timer_ns() - t0);
+            atomicAdd(acc + 1, (unsigned long long)clock64() - c0);
+            atomicAdd(acc + 2, 1ull);
+        }
+    }
+};
 
 // Bounded wait.  Returns false when the block is aborting (this wait ran out, or another did).
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, SharedControl *ctl, int32_t *status,

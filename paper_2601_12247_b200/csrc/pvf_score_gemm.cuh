@@ -91,6 +91,8 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     // Everything above touched no global memory: it may overlap the tail of the kernel before this
     // one in the stream.  From here on the hidden states are read and the partial states written.
     pvf_grid_dependency_wait();
+    LaunchClock launch_clock;
+    launch_clock.begin();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -190,6 +192,7 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     __syncthreads();
     // Only now may the next kernel's blocks become resident: while they wait for this grid they would
     // share the SM with the MMA and epilogue warps.
+    launch_clock.end(args.clock_acc);
     pvf_launch_dependents();
     if (warp == 1) {
         tc_fence_after_sync();

@@ -89,6 +89,8 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
     pvf_grid_dependency_wait();
+    LaunchClock launch_clock;
+    launch_clock.begin();
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -232,6 +234,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
 
     tc_fence_before_sync();
     __syncthreads();
+    launch_clock.end(args.clock_acc);
     pvf_launch_dependents();
     if (warp == 1) {
         tc_fence_after_sync();

@@ -210,6 +210,8 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
     pvf_grid_dependency_wait();
+    LaunchClock launch_clock;
+    launch_clock.begin();
 
     SwapLoopArgs la;
     la.tiles_addr = tiles_addr; la.stage_bytes = stage_bytes; la.h0_bytes = h0_bytes; la.h1_bytes = h1_bytes;
@@ -313,6 +315,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     tc_fence_before_sync();
     __syncthreads();
     cluster_sync_all();
+    launch_clock.end(args.clock_acc);
     pvf_launch_dependents();
     if (warp == 1) {
         tc_fence_after_sync();

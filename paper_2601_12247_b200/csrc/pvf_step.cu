@@ -596,7 +596,7 @@ int pvf_draft_step(pvf_ctx *ctx, const pvf_params *params, const void *hidden, i
         return PVF_ERR_INVALID;
     int parts = 0;
     if (M > 0) {
-        const int rc = pvf_score_partials(ctx, hidden, M, &parts, stream);
+        const int rc = pvf_score_partials(ctx, hidden, M, &parts, 0, stream);
         if (rc != PVF_OK) return rc;
     }
     const int share = merge_share(M, n_seq, parts);
@@ -626,7 +626,7 @@ int pvf_verify_step(pvf_ctx *ctx, const pvf_params *params, const void *hidden_v
         return PVF_ERR_INVALID;
     int parts = 0;
     if (Mv > 0) {
-        const int rc = pvf_score_partials(ctx, hidden_v, Mv, &parts, stream);
+        const int rc = pvf_score_partials(ctx, hidden_v, Mv, &parts, 1, stream);
         if (rc != PVF_OK) return rc;
         const int share = merge_share(Mv, n_seq, parts);
         return launch_result(pvf_launch(pvf_verify_kernel<true>, dim3(n_seq * share), dim3(kThreads), 0, (cudaStream_t)stream,

@@ -52,6 +52,10 @@ def test_default_workload_line():
     assert r["timed_every_nth_step"] == 8 and d["repeats"] >= 20      # 24 steps of a third of a millisecond: many blocks
     assert d["clocks"]["samples"] >= 10 and d["clocks"]["sm_mhz"] > 0
     assert r["sm_cycles_per_launch"] == pytest.approx(r["avg_launch_us"] * d["clocks"]["sm_mhz"], rel=1e-9)
+    for item in r["per_row_count"]:                               # the kernels' own clock: every launch of the region counted
+        assert item["device_launches"] == d["steps"] * d["repeats"] and 500 < item["device_sm_mhz"] <= d["clocks"]["sm_max_mhz"] + 1
+        assert item["device_sm_cycles"] == pytest.approx(item["device_kernel_us"] * item["device_sm_mhz"], rel=1e-6)
+        assert 0.8 * item["avg_launch_us"] < item["device_kernel_us"] <= 1.02 * item["avg_launch_us"]
     e = d["e2e"]
     assert e["unit"] == d["unit"] and e["h2d_bytes_per_step"] > 2 * 30 * 4096 * 2 and e["d2h_bytes_per_step"] > 0
     assert e["value"] < d["value"]                                   # host copies inside the timed region
