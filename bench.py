@@ -37,15 +37,17 @@ UNIT = "positions/s"
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one pass over W ("wave") of each projection
 # kernel, from the ncu captures summarised under profiles/ (None = not captured since the kernel last changed).
-# The streaming and swapped paired kernels' launches are one pass; launches of the GEMM kernels scale the
-# captured per-pass traffic by their number of passes.
+# The streaming and swapped paired kernels' launches are one pass. A launch of the paired kernel with several
+# waves (18 row tiles x 4 pairs each at the LLaDA shape) was captured at 3 waves; its traffic grows with the
+# number of waves, so larger launches scale the per-wave figure.
 NCU_TRAFFIC_PER_WAVE = {
-    "pvf_score_stream_kernel": 1.04217e9,
-    "pvf_score_gemm_kernel": 1.277e9,
-    "pvf_score_gemm_pair_kernel": 1.0490e9,
-    "pvf_score_swap_pair_kernel": 1.0504e9,
+    "pvf_score_stream_kernel": 1.04026e9,
+    "pvf_score_gemm_kernel": None,
+    "pvf_score_gemm_pair_kernel": 1.04176e9,
+    "pvf_score_swap_pair_kernel": 1.04166e9,
 }
-NCU_TRAFFIC_SWAP_WIDE = 1.0572e9          # the swapped paired kernel above 256 rows (two column groups)
+NCU_TRAFFIC_SWAP_WIDE = 1.0425e9          # the swapped paired kernel above 256 rows (two column groups)
+NCU_TRAFFIC_PAIR_MULTI_WAVE = 1.908e9     # the paired kernel, per wave, in launches of several waves
 
 
 def load_peaks():
@@ -236,8 +238,14 @@ def roofline_of(pairs, ctx, V, D, peaks, sm_mhz, event_every):
 
     def launch_traffic(rows):
         name = ctx.score_kernel_name(rows)
-        per_wave = NCU_TRAFFIC_SWAP_WIDE if (name == "pvf_score_swap_pair_kernel" and rows > 256) else NCU_TRAFFIC_PER_WAVE.get(name)
-        return None if per_wave is None else per_wave * ctx.score_plan(rows)["waves"]
+        waves = ctx.score_plan(rows)["waves"]
+        if name == "pvf_score_swap_pair_kernel" and rows > 256:
+            per_wave = NCU_TRAFFIC_SWAP_WIDE
+        elif name == "pvf_score_gemm_pair_kernel" and waves > 1:
+            per_wave = NCU_TRAFFIC_PAIR_MULTI_WAVE
+        else:
+            per_wave = NCU_TRAFFIC_PER_WAVE.get(name)
+        return None if per_wave is None else per_wave * waves
     per_launch = [launch_traffic(r) for _, r in durs]
     traffic = sum(per_launch) / n if per_launch and all(x is not None for x in per_launch) else None
     by_rows = {}

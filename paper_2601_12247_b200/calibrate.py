@@ -2,15 +2,17 @@
 (Appendix, "Planning Token Set Construction").
 
 The canvas is decoded with the confidence-threshold base rule alone.  At every step the calibration candidates
-(non-base masked positions of the working block whose confidence lies in the calibration band, any top-1 token,
-the most confident first, at most ``budget`` per sequence) are measured: one planning branch each, scored with
+(non-base masked positions of the working block whose confidence lies in the calibration band, any top-1 token)
+are measured -- all of them, as in the paper, when ``budget`` is at least the block size (the default; the library
+takes budgets up to 64); a smaller budget keeps the most confident ones only, which is a caller's choice that departs
+from the paper: one planning branch each, scored with
 entropies, checked with pvf_verify, and their events added to the per-token statistics with
 pvf_calib_accumulate.  The branches are never committed.  pvf_calib_filter turns the statistics into the
 vocabulary.  The transformer is replaced by the seeded generator of ``synth`` (the paper's calibration corpora
 are not available here): this is a harness around the library that shows the whole path and reports its
 kernel time.
 
-    python -m paper_2601_12247_b200.calibrate [--n-seq 32] [--gen-len 256] [--block 32] [--budget 8]
+    python -m paper_2601_12247_b200.calibrate [--n-seq 32] [--gen-len 256] [--block 32] [--budget min(64, block)]
 """
 from __future__ import annotations
 
@@ -93,12 +95,15 @@ def main():
     ap.add_argument("--n-seq", type=int, default=32)
     ap.add_argument("--gen-len", type=int, default=256)
     ap.add_argument("--block", type=int, default=32)
-    ap.add_argument("--budget", type=int, default=8)
+    ap.add_argument("--budget", type=int, default=None,
+                    help="candidates measured per sequence and step; default min(64, block): every candidate of the band")
     ap.add_argument("--n-tokens", type=int, default=64, help="targets are drawn from this many token ids, so that tokens repeat")
     ap.add_argument("--n-min", type=int, default=5)
     ap.add_argument("--m-min", type=int, default=2)
     ap.add_argument("--seed", type=int, default=1006)
     args = ap.parse_args()
+    if args.budget is None:
+        args.budget = min(64, args.block)
     dev = torch.device("cuda:0")
     w_bits = synth.make_w(args.seed, args.vocab, args.hidden)
     pool = synth.make_plan_ids(args.seed, args.vocab, args.n_tokens)

@@ -123,16 +123,23 @@ def test_exploration_loop_state_by_state(mode):
 
 
 @pytest.mark.gpu
-def test_calibration_trajectory_matches_oracle():
+@pytest.mark.parametrize("K,band,min_widest", [(8, (None, 0.6), 1), (32, (0.02, 0.9), 9)])
+def test_calibration_trajectory_matches_oracle(K, band, min_widest):
+    # K = 8 with a band a little wider than the paper's; and K = 32 = the block size with a band so wide that more
+    # than 8 rows of a sequence fall into it at once: with the budget at least the block size every candidate of
+    # C_t^cal is measured, which is the paper's rule (Appendix, "Calibration trajectory") -- the oracle runs with the
+    # same budget, which then never binds.
     from oracle import calib as ocal
     from paper_2601_12247_b200 import calibrate
-    V, D, B, L, S, seed, K = 4096, 256, 4, 64, 32, 1006, 8
+    V, D, B, L, S, seed = 4096, 256, 4, 64, 32, 1006
     w = synth.make_w(seed, V, D)
     pool = synth.make_plan_ids(seed, V, 24)
     tg = synth.loop_targets(seed, V, B, L, pool, 1.0, avoid=V - 1)
     mask = V - 1
     cal = binding.default_calib_params()
-    cal.tau_cal_hi = 0.6                                     # a wider band than the paper's: more events in a tiny run
+    if band[0] is not None:
+        cal.tau_cal_lo = band[0]
+    cal.tau_cal_hi = band[1]                                 # a wider band than the paper's: more events in a tiny run
     want = ocal.calibrate(synth, w, tg, seed, L, S, 0.9, cal.tau_cal_lo, cal.tau_cal_hi, K, mask, trace=True)
     ctx = make_ctx(w, [], B * S * (2 + K), B, K)
     trace = []
@@ -156,6 +163,8 @@ def test_calibration_trajectory_matches_oracle():
                 assert abs(vig[e["seq"], e["j"] - 1] - e["VIG"]) <= 2e-3       # entropies within 1e-3 on both branches
         assert np.array_equal(g["y"], o["y"])
     assert want["n_events"] > 0
+    widest = max(int(o["select"]["n_drafts"].max()) for o in want["history"])
+    assert min_widest <= widest <= K and (K < S or widest < K)              # K = S: the budget never binds
     if clean:
         st = to_np(got["stats"])
         assert got["steps"] == want["steps"] and got["n_events"] == want["n_events"]
