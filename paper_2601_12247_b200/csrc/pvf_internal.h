@@ -163,8 +163,8 @@ __device__ __forceinline__ void pvf_state_merge(float4 &a, const float4 b)
 // Final merge of rows [row_begin, row_end) by the warps of a block, or of a grid of such blocks (all threads call it;
 // `warp` / `n_warps` = this warp's index among the warps that share the row range).  A row's `parts` partial states
 // are folded by g = min(32, parts rounded up to a power of two) neighbouring lanes -- lane l takes states l, l + g,
-// ... in turn, then the lanes fold pairwise: an order fixed by `parts` alone, so results are identical from run to
-// run -- and the row's first lane writes token, confidence = 1 / (1 + y), entropy = ln(1 + y) - z / (1 + y) and
+// ... five at a time, folds them pairwise, then the lanes fold pairwise: an order fixed by `parts` alone, so results
+// are identical from run to run -- and the row's first lane writes token, confidence = 1 / (1 + y), entropy = ln(1 + y) - z / (1 + y) and
 // planning-vocabulary membership (Section 3: y^, p, H; Section 4.1: y^ in P^plan).  ent and in_plan may be NULL.
 // A warp works on kMergeRowsInFlight groups of 32 / g rows at once and fetches up to kMergeStatesInFlight states per
 // lane and row before it merges any (the merge is a chain of memory round trips otherwise).  No shared memory and
@@ -199,22 +199,39 @@ __device__ __forceinline__ void pvf_merge_rows(const float4 *__restrict__ partia
                 for (int k = 0; k < kMergeStatesInFlight; ++k)
                     v[r][k] = (row < row_end && i0 + k * g < parts) ? __ldg(partials + (size_t)row * parts + i0 + k * g) : none;
             }
+            // The states a lane holds are folded pairwise -- (0 1)(2 3), then the pairs, then the fifth -- and the rows
+            // side by side: a merge is a chain of some sixty dependent instructions, and with two warps per
+            // scheduler nothing else hides their latency.
+            static_assert(kMergeStatesInFlight == 5, "the fold below is written out for five states");
 #pragma unroll
-            for (int r = 0; r < kMergeRowsInFlight; ++r)
+            for (int r = 0; r < kMergeRowsInFlight; ++r) {
+                pvf_state_merge(v[r][0], v[r][1]);
+                pvf_state_merge(v[r][2], v[r][3]);
+            }
 #pragma unroll
-                for (int k = 0; k < kMergeStatesInFlight; ++k) pvf_state_merge(acc[r], v[r][k]);
+            for (int r = 0; r < kMergeRowsInFlight; ++r) pvf_state_merge(v[r][0], v[r][2]);
+#pragma unroll
+            for (int r = 0; r < kMergeRowsInFlight; ++r) pvf_state_merge(v[r][0], v[r][4]);
+#pragma unroll
+            for (int r = 0; r < kMergeRowsInFlight; ++r) pvf_state_merge(acc[r], v[r][0]);
+        }
+#pragma unroll 1
+        for (int o = 1; o < g; o <<= 1) {                       // lane l absorbs lane l + o of its row
+            float4 other[kMergeRowsInFlight];
+#pragma unroll
+            for (int r = 0; r < kMergeRowsInFlight; ++r) {
+                other[r].x = __shfl_down_sync(0xffffffffu, acc[r].x, o, g);
+                other[r].y = __shfl_down_sync(0xffffffffu, acc[r].y, o, g);
+                other[r].z = __shfl_down_sync(0xffffffffu, acc[r].z, o, g);
+                other[r].w = __shfl_down_sync(0xffffffffu, acc[r].w, o, g);
+            }
+            if ((gl & (2 * o - 1)) == 0) {
+#pragma unroll
+                for (int r = 0; r < kMergeRowsInFlight; ++r) pvf_state_merge(acc[r], other[r]);
+            }
         }
 #pragma unroll
         for (int r = 0; r < kMergeRowsInFlight; ++r) {
-#pragma unroll 1
-            for (int o = 1; o < g; o <<= 1) {                   // lane l absorbs lane l + o of its row
-                float4 other;
-                other.x = __shfl_down_sync(0xffffffffu, acc[r].x, o, g);
-                other.y = __shfl_down_sync(0xffffffffu, acc[r].y, o, g);
-                other.z = __shfl_down_sync(0xffffffffu, acc[r].z, o, g);
-                other.w = __shfl_down_sync(0xffffffffu, acc[r].w, o, g);
-                if ((gl & (2 * o - 1)) == 0) pvf_state_merge(acc[r], other);
-            }
             const int row = row0 + r * rows_per_pass + sub;
             if (gl == 0 && row < row_end) {
                 // A row of non-finite logits never sets a maximum: its outputs are unspecified, but the token stays a

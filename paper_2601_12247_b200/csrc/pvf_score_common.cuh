@@ -185,6 +185,13 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"((unsigned long long)map), "r"(bar), "r"(x), "r"(y), "l"(policy) : "memory");
 }
 
+// Asks TMA to bring the box at (x, y) into L2 (no shared memory, no barrier: a hint).
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap *map, int x, int y, uint64_t policy)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile.L2::cache_hint [%0, {%1, %2}], %3;"
+                 ::"l"((unsigned long long)map), "r"(x), "r"(y), "l"(policy) : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 

@@ -24,6 +24,7 @@ constexpr int kStreamWBytes = kStreamTileN * kRowBytes;             // 32 KiB
 constexpr int kStreamStageBytes = kStreamHBytes + kStreamWBytes;
 constexpr int kStreamTmemCols = 128;                                // 2 buffers x 2 slices x 32 columns
 constexpr int kStreamControlBytes = 512;
+constexpr int kStreamL2PrefetchSteps = 16;                          // W boxes (up to 32 KB each) asked into L2 before the wait
 constexpr int kStreamIssuers = 2;                                   // MMA-issuing threads (one per vocabulary slice)
 constexpr int kStreamSecondIssuerWarp = 6;
 constexpr int kStreamThreads = 224;                                 // producer, issuer, 4 epilogue warps, issuer
@@ -88,6 +89,40 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
+    pvf_launch_dependents();
+
+    // W is a constant of the context: nothing the kernels before this one in the stream do can change it.  The
+    // producer therefore starts the W tiles of the first ring of stages BEFORE the grid-dependency wait (the hidden
+    // states, which the predecessor may still be writing, follow after it): the weight stream of this launch starts
+    // on every SM the previous launch has left, while its slowest blocks and the decision kernel between the two
+    // launches are still running.  The ring holds 192 KB of the block's 7 MB; the SM would then idle until the wait
+    // returns (the spread of the previous launch's block ends plus the decision kernel: 15 .. 20 us), so the W boxes
+    // that follow are asked into L2 (a hint, evict-first like the loads themselves), where the loads after the wait
+    // find them.
+    ArmedStages armed;
+    int prefetched = 0;
+    if (threadIdx.x == 0) {
+        const uint64_t w_policy = w_evict_first_policy();
+        int ahead = 0;                                               // W boxes asked into L2 beyond the ring
+        for (int tile = 0; tile < n_tiles && (prefetched < kStreamStages || ahead < kStreamL2PrefetchSteps); ++tile) {
+            int tu0, tun;
+            split.tile(tile, &tu0, &tun);
+            const uint32_t bytes = (uint32_t)args.a_rows * kRowBytes + (uint32_t)tun * kUnitBytes;
+            for (int step = 0; step < k_steps && (prefetched < kStreamStages || ahead < kStreamL2PrefetchSteps); ++step) {
+                if (prefetched < kStreamStages) {
+                    const uint32_t full = smem_u32(&ctl->full[prefetched]);
+                    mbar_arrive_expect_tx(full, bytes);              // the stage's H panel and W tile
+                    armed.note(prefetched, 0u);
+                    load_w_tile<true>(tiles_addr + prefetched * kStreamStageBytes + kStreamHBytes, tm_w, full, step * kBlockK, tu0,
+                                      tun, w_policy);
+                    ++prefetched;
+                } else {
+                    tma_prefetch_l2_2d(&tm_w.size[tun - 1], step * kBlockK, tu0 * kUnit, w_policy);
+                    ++ahead;
+                }
+            }
+        }
+    }
     pvf_grid_dependency_wait();
     LaunchClock launch_clock;
     launch_clock.begin();
@@ -97,21 +132,25 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
-            ArmedStages armed;
+            int issued = 0;
             const uint64_t w_policy = w_evict_first_policy();         // one wave, one row tile: W is read once
             bool alive = true;
             for (int tile = 0; tile < n_tiles && alive; ++tile) {
                 int tu0, tun;
                 split.tile(tile, &tu0, &tun);
                 const uint32_t bytes = (uint32_t)args.a_rows * kRowBytes + (uint32_t)tun * kUnitBytes;
-                for (int step = 0; step < k_steps; ++step) {
-                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                for (int step = 0; step < k_steps; ++step, ++issued) {
                     const uint32_t full = smem_u32(&ctl->full[stage]);
                     const uint32_t h_dst = tiles_addr + stage * kStreamStageBytes;
-                    mbar_arrive_expect_tx(full, bytes);
-                    armed.note(stage, phase);
-                    tma_load_2d(h_dst, &tm_h, full, step * kBlockK, 0);
-                    load_w_tile<true>(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, w_policy);
+                    if (issued < prefetched) {                           // armed, W tile on its way: the H panel is left
+                        tma_load_2d(h_dst, &tm_h, full, step * kBlockK, 0);
+                    } else {
+                        if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                        mbar_arrive_expect_tx(full, bytes);
+                        armed.note(stage, phase);
+                        tma_load_2d(h_dst, &tm_h, full, step * kBlockK, 0);
+                        load_w_tile<true>(h_dst + kStreamHBytes, tm_w, full, step * kBlockK, tu0, tun, w_policy);
+                    }
                     if (++stage == kStreamStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -235,7 +274,6 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     tc_fence_before_sync();
     __syncthreads();
     launch_clock.end(args.clock_acc);
-    pvf_launch_dependents();
     if (warp == 1) {
         tc_fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kStreamTmemCols) : "memory");

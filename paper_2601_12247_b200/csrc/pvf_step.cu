@@ -194,6 +194,19 @@ __device__ __forceinline__ void select_block(int b, int n_seq, const int32_t *__
         rt = kt > 0 ? 2 : 0;
     }
     for (int j = kt + threadIdx.x; j < K; j += kThreads) draft_rows[(size_t)b * K + j] = -1;
+    if (n_seq == 1 && r0 == 0) {
+        // One sequence: its list is where it belongs and the offsets are its lengths -- no ticket, no fences, no
+        // packing (four dependent round trips to L2, 3 .. 4 us of a batch-1 step).
+        if (threadIdx.x == 0) {
+            n_drafts[0] = kt;
+            route[0] = (uint8_t)rt;
+            rem_off[0] = 0;
+            rem_off[1] = n_rem;
+            v_off[0] = 0;
+            v_off[1] = kt > 0 ? (1 + kt) * n_rem : 0;
+        }
+        return;
+    }
     if (threadIdx.x == 0) {
         n_drafts[b] = kt;
         route[b] = (uint8_t)rt;
