@@ -121,14 +121,50 @@ __device__ __forceinline__ void wave_boundary(uint32_t *arrivals, unsigned targe
     }
 }
 
+// Before the grid-dependency wait of a launch of one wave (W is read once): the producer arms the first ring of
+// stages and starts this block's half of their W tiles, then asks the W boxes that follow into L2.  W is a constant
+// of the context -- nothing earlier in the stream can change it -- so the weight stream of this launch starts on
+// every SM the previous launch has left while the rest of it, and the decision kernel between the two, still run.
+// Returns the number of stages started; pair_produce then only adds their hidden-state tiles.
+constexpr int kPairL2PrefetchSteps = 16;
+__device__ __forceinline__ int pair_prefetch_w(const ScoreArgs &args, const WMaps &tm_w, SharedControl *ctl, uint32_t tiles_addr,
+                                               int pair, uint32_t rank, int k_steps, ArmedStages &armed)
+{
+    int s_tile, q, u0, u1;
+    if (!pair_wave_work(args, pair, 0, &s_tile, &q, &u0, &u1)) return 0;
+    const TileSplit split(u0, u1, kPairUnitsPerTile);
+    const uint64_t w_policy = w_evict_first_policy();
+    int started = 0, ahead = 0;
+    for (int tile = 0; tile < split.n_tiles && (started < kPairStages || ahead < kPairL2PrefetchSteps); ++tile) {
+        int tu0, tun;
+        split.tile(tile, &tu0, &tun);
+        const uint32_t bytes = 2u * ((uint32_t)kPairABytes + (uint32_t)tun * kUnitBytes);
+        const int w_row = tu0 * kPairUnit + (int)rank * tun * kUnit;
+        for (int step = 0; step < k_steps && (started < kPairStages || ahead < kPairL2PrefetchSteps); ++step) {
+            if (started < kPairStages) {
+                const uint32_t full = smem_u32(&ctl->full[started]);
+                if (rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(started, 0u); }
+                tma_load_2d_pair_hint(tiles_addr + started * kPairStageBytes + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row,
+                                      w_policy);
+                ++started;
+            } else {
+                tma_prefetch_l2_2d(&tm_w.size[tun - 1], step * kBlockK, w_row, w_policy);
+                ++ahead;
+            }
+        }
+    }
+    return started;
+}
+
 // The TMA producer's loop (one thread per block).  kReadOnce: W is read exactly once by the launch (evict-first hint).
+// `started` stages (of wave 0) are armed and have their W tiles on the way already (pair_prefetch_w).
 template <bool kReadOnce>
 __device__ __forceinline__ void pair_produce(const ScoreArgs &args, const CUtensorMap &tm_h, const WMaps &tm_w, SharedControl *ctl,
-                                             uint32_t tiles_addr, int pair, uint32_t rank, int k_steps)
+                                             uint32_t tiles_addr, int pair, uint32_t rank, int k_steps, int started, ArmedStages armed)
 {
     int stage = 0;
     uint32_t phase = 0;
-    ArmedStages armed;                                                       // even block: it arms full[]
+    int issued = 0;
     const uint64_t w_policy = kReadOnce ? w_evict_first_policy() : 0ull;
     bool alive = true;
     for (int w = 0; w < args.waves && alive; ++w) {
@@ -143,14 +179,18 @@ __device__ __forceinline__ void pair_produce(const ScoreArgs &args, const CUtens
             split.tile(tile, &tu0, &tun);
             const uint32_t bytes = 2u * ((uint32_t)kPairABytes + (uint32_t)tun * kUnitBytes);   // both blocks
             const int w_row = tu0 * kPairUnit + (int)rank * tun * kUnit;                        // this block's half
-            for (int step = 0; step < k_steps; ++step) {
-                if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+            for (int step = 0; step < k_steps; ++step, ++issued) {
                 const uint32_t full = smem_u32(&ctl->full[stage]);
                 const uint32_t a_dst = tiles_addr + stage * kPairStageBytes;
-                if (rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
-                tma_load_2d_pair(a_dst, &tm_h, full, step * kBlockK, row0);
-                if (kReadOnce) tma_load_2d_pair_hint(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
-                else tma_load_2d_pair(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
+                if (issued < started) {                                      // armed, W half on its way: the H tile is left
+                    tma_load_2d_pair(a_dst, &tm_h, full, step * kBlockK, row0);
+                } else {
+                    if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, args.status)) { alive = false; break; }
+                    if (rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
+                    tma_load_2d_pair(a_dst, &tm_h, full, step * kBlockK, row0);
+                    if (kReadOnce) tma_load_2d_pair_hint(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
+                    else tma_load_2d_pair(a_dst + kPairABytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row);
+                }
                 if (++stage == kPairStages) { stage = 0; phase ^= 1u; }
             }
         }
@@ -202,6 +242,12 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     cluster_sync_all();                                                  // the peer's barriers exist before anything signals them
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
+    ArmedStages armed;                                                   // even block: it arms full[]
+    int started = 0;
+    if (args.w_once) {
+        pvf_launch_dependents();                                         // one wave: the next launch may move in as this one leaves
+        if (threadIdx.x == 0) started = pair_prefetch_w(args, tm_w, ctl, tiles_addr, pair, rank, k_steps, armed);
+    }
     pvf_grid_dependency_wait();
     LaunchClock launch_clock;
     launch_clock.begin();
@@ -209,8 +255,8 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (one per block)
         if (lane == 0) {
-            if (args.w_once) pair_produce<true>(args, tm_h, tm_w, ctl, tiles_addr, pair, rank, k_steps);
-            else pair_produce<false>(args, tm_h, tm_w, ctl, tiles_addr, pair, rank, k_steps);
+            if (args.w_once) pair_produce<true>(args, tm_h, tm_w, ctl, tiles_addr, pair, rank, k_steps, started, armed);
+            else pair_produce<false>(args, tm_h, tm_w, ctl, tiles_addr, pair, rank, k_steps, 0, armed);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even block only)
@@ -309,7 +355,7 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     __syncthreads();
     cluster_sync_all();                                                  // neither block leaves while the other may still signal it
     launch_clock.end(args.clock_acc);
-    pvf_launch_dependents();
+    if (!args.w_once) pvf_launch_dependents();                           // several waves: the next kernel could only wait beside this one
     if (warp == 1) {
         tc_fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kPairTmemCols) : "memory");

@@ -75,15 +75,45 @@ struct SwapLoopArgs {
     uint32_t rank;
 };
 
+// Before the grid-dependency wait (W is a constant of the context, see the paired GEMM kernel's pair_prefetch_w): arm
+// the first ring of stages, start this block's W tiles of them, ask the boxes that follow into L2.  Returns the
+// number of stages started; swap_produce then only adds their hidden-state tiles.
+constexpr int kSwapL2PrefetchSteps = 16;
+__device__ __forceinline__ int swap_prefetch_w(const SwapLoopArgs &a, const TileSplit &split, SharedControl *ctl, const WMaps &tm_w,
+                                               bool wide, ArmedStages &armed)
+{
+    const uint64_t w_policy = w_evict_first_policy();
+    int started = 0, ahead = 0;
+    for (int tile = 0; tile < a.n_tiles && (started < a.n_stages || ahead < kSwapL2PrefetchSteps); ++tile) {
+        int tu0, tun;
+        split.tile(tile, &tu0, &tun);
+        const uint32_t bytes = 2u * ((uint32_t)tun * kUnitBytes + a.h0_bytes + (wide ? a.h1_bytes : 0u));
+        const int w_row = tu0 * kPairUnit + (int)a.rank * tun * kUnit;
+        for (int step = 0; step < a.k_steps && (started < a.n_stages || ahead < kSwapL2PrefetchSteps); ++step) {
+            if (started < a.n_stages) {
+                const uint32_t full = smem_u32(&ctl->full[started]);
+                if (a.rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(started, 0u); }
+                tma_load_2d_pair_hint(a.tiles_addr + (uint32_t)started * a.stage_bytes, &tm_w.size[tun - 1], full, step * kBlockK, w_row,
+                                      w_policy);
+                ++started;
+            } else {
+                tma_prefetch_l2_2d(&tm_w.size[tun - 1], step * kBlockK, w_row, w_policy);
+                ++ahead;
+            }
+        }
+    }
+    return started;
+}
+
 template <bool kWide>
 __device__ __forceinline__ void swap_produce(const SwapLoopArgs &a, const TileSplit &split, SharedControl *ctl,
                                              const CUtensorMap *tm_h, const CUtensorMap *tm_h1, const WMaps &tm_w,
-                                             int32_t *status)
+                                             int32_t *status, int started, ArmedStages armed)
 {
     int stage = 0;
     uint32_t phase = 0;
+    int issued = 0;
     bool alive = true;
-    ArmedStages armed;
     const uint64_t w_policy = w_evict_first_policy();            // one wave, one row tile: W is read once
     const int row0 = (int)a.rank * (a.n0 / 2);                                      // this block's half of each group's rows
     const int row1 = a.n0 + (int)a.rank * (a.n1 / 2);
@@ -92,12 +122,14 @@ __device__ __forceinline__ void swap_produce(const SwapLoopArgs &a, const TileSp
         split.tile(tile, &tu0, &tun);
         const uint32_t bytes = 2u * ((uint32_t)tun * kUnitBytes + a.h0_bytes + (kWide ? a.h1_bytes : 0u));   // both blocks
         const int w_row = tu0 * kPairUnit + (int)a.rank * tun * kUnit;                                        // this block's entries
-        for (int step = 0; step < a.k_steps; ++step) {
-            if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, status)) { alive = false; break; }
+        for (int step = 0; step < a.k_steps; ++step, ++issued) {
             const uint32_t full = smem_u32(&ctl->full[stage]);
             const uint32_t w_dst = a.tiles_addr + (uint32_t)stage * a.stage_bytes;
-            if (a.rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
-            tma_load_2d_pair_hint(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
+            if (issued >= started) {                                                // else: armed, W tile on its way already
+                if (!mbar_wait(smem_u32(&ctl->empty[stage]), phase ^ 1u, ctl, status)) { alive = false; break; }
+                if (a.rank == 0) { mbar_arrive_expect_tx(full, bytes); armed.note(stage, phase); }
+                tma_load_2d_pair_hint(w_dst, &tm_w.size[tun - 1], full, step * kBlockK, w_row, w_policy);
+            }
             tma_load_2d_pair(w_dst + kSwapWBytes, tm_h, full, step * kBlockK, row0);
             if (kWide) tma_load_2d_pair(w_dst + kSwapWBytes + a.h0_bytes, tm_h1, full, step * kBlockK, row1);
             if (++stage == a.n_stages) { stage = 0; phase ^= 1u; }
@@ -209,19 +241,23 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     cluster_sync_all();
     tc_fence_after_sync();
     const uint32_t tmem_base = ctl->tmem_base;
-    pvf_grid_dependency_wait();
-    LaunchClock launch_clock;
-    launch_clock.begin();
-
     SwapLoopArgs la;
     la.tiles_addr = tiles_addr; la.stage_bytes = stage_bytes; la.h0_bytes = h0_bytes; la.h1_bytes = h1_bytes;
     la.tmem_base = tmem_base; la.n0 = n0; la.n1 = n1; la.n_stages = n_stages; la.n_tiles = n_tiles; la.k_steps = k_steps;
     la.n_bufs = n_bufs; la.rank = rank;
+    pvf_launch_dependents();                                             // one wave: the next launch may move in as this one leaves
+    ArmedStages armed;                                                   // even block: it arms full[]
+    int started = 0;
+    if (threadIdx.x == 0) started = swap_prefetch_w(la, split, ctl, tm_w, n1 != 0, armed);
+    pvf_grid_dependency_wait();
+    LaunchClock launch_clock;
+    launch_clock.begin();
+
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer (one per block)
         if (lane == 0) {
-            if (n1 == 0) swap_produce<false>(la, split, ctl, &tm_h, &tm_h1, tm_w, args.status);
-            else swap_produce<true>(la, split, ctl, &tm_h, &tm_h1, tm_w, args.status);
+            if (n1 == 0) swap_produce<false>(la, split, ctl, &tm_h, &tm_h1, tm_w, args.status, started, armed);
+            else swap_produce<true>(la, split, ctl, &tm_h, &tm_h1, tm_w, args.status, started, armed);
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (even block only)
@@ -316,7 +352,6 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     __syncthreads();
     cluster_sync_all();
     launch_clock.end(args.clock_acc);
-    pvf_launch_dependents();
     if (warp == 1) {
         tc_fence_after_sync();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kSwapTmemCols) : "memory");
