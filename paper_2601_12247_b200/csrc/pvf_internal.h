@@ -78,10 +78,14 @@ int pvf_score_init(pvf_ctx *ctx);   // tensor maps of W, kernel attributes
 int pvf_score_partials(pvf_ctx *ctx, const void *hidden, int32_t M, int *parts, int clock_slot, void *stream);
 
 // Programmatic dependent launch.  Every kernel of the library is launched with pvf_launch and runs
-//     <set-up that touches no global memory>; pvf_launch_dependents(); pvf_grid_dependency_wait();
-// before its first global access, on every thread.  The wait returns once the kernel before it in
-// the stream has completed and its writes are visible, so stream order is kept; what overlaps is the
-// launch latency and set-up of a kernel with the tail of its predecessor.
+//     <set-up>; pvf_launch_dependents(); pvf_grid_dependency_wait();
+// before it reads anything an earlier kernel may have written, or writes anything, on every thread.  The wait returns
+// once the kernel before it in the stream has completed and its writes are visible, so stream order is kept; what
+// overlaps is the launch latency and set-up of a kernel with the tail of its predecessor.  Two departures, both in
+// the projection kernels: (1) their set-up includes reads of W -- the LM-head weights are a constant of the context,
+// which no kernel in the stream writes -- so in launches of one wave the first tiles of W are on their way, and
+// further ones asked into L2, before the wait; (2) launches of several waves let their dependents in at their end
+// only, since all those could do earlier is wait beside blocks that run for milliseconds.
 #ifdef __CUDACC__
 __device__ __forceinline__ void pvf_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pvf_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

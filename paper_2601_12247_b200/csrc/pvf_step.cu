@@ -6,12 +6,14 @@
 // merge of its partial softmax states as their first phase:
 //     pvf_draft_kernel            merge (the sequence's own rows) + base commit + draft proposal
 //     pvf_verify_kernel<true>     merge (the sequence's rows of the verification pass) + acceptance check
-// so that a step is four launches.  These kernels keep to a few dozen registers and about a kilobyte of shared memory:
-// they are launched (programmatic dependent launch) while the projection kernel still runs, and only fit beside its
-// blocks -- which fill an SM's shared memory and two thirds of its registers -- if they stay that small; a version
-// that staged the merge through 96 KB of shared memory, or held 20 states per thread in registers, could not become
-// resident before the projection ended and was 4 .. 6 us per step slower.  Pointers that one phase of a kernel writes and a later phase reads carry no
-// __restrict__ / read-only qualifier in the shared device functions.
+// so that a step is four launches.  These kernels keep to a few dozen registers and about a kilobyte of shared memory.
+// Measured with %globaltimer stamps: a block of theirs becomes resident on the first SM that a block of the running
+// projection leaves, some ten microseconds before its grid-dependency wait returns, and the block of the NEXT
+// projection that takes over that SM (it starts fetching weights before its own wait) must fit beside it -- a
+// projection block fills an SM's shared memory and two thirds of its registers.  A version that staged the merge
+// through 96 KB of shared memory, or held 20 states per thread in registers, was 4 .. 6 us per step slower.  Pointers
+// that one phase of a kernel writes and a later phase reads carry no __restrict__ / read-only qualifier in the shared
+// device functions.
 #include "pvf_internal.h"
 
 namespace {
