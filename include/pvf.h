@@ -105,7 +105,10 @@ size_t pvf_workspace_bytes(const pvf_shape *shape);
 
 /*
  * Create a context.
- *   w_head          device, bf16 [vocab][hidden] row-major, 16-byte aligned: the LM head.  Kept.
+ *   w_head          device, bf16 [vocab][hidden] row-major, 16-byte aligned: the LM head.  Kept, and treated as
+ *                   constant until pvf_destroy: the scoring kernels start reading it before the work queued
+ *                   ahead of them on their stream has completed.  To change the weights, synchronise the
+ *                   streams that use the context first, then write them (or create a new context).
  *   plan_ids_host   HOST, n_plan token ids of the planning vocabulary P^plan (Section 3; any order,
  *                   duplicates allowed, each in [0, vocab)).  Copied into a device bitmap during the
  *                   call (this call synchronises the device once).
@@ -423,7 +426,8 @@ int pvf_verify_step_host(pvf_ctx *ctx, const pvf_params *params, const void *hid
  * do not fit -- more than 221 rows -- this entry point takes the kernel pvf_score uses outside that window:
  * same arithmetic, results equal within the accumulation order.)
  *
- *   w_head       device, bf16 [vocab][hidden_size] row-major, 16-byte aligned
+ *   w_head       device, bf16 [vocab][hidden_size] row-major, 16-byte aligned; not written by work still queued
+ *                on the stream when the call is made (the kernels start reading it before that work is done)
  *   hidden       device, bf16 [M][hidden_size], 16-byte aligned; hidden_size a multiple of 8
  *   M            at most PVF_STATIC_MAX_ROWS; larger M returns PVF_ERR_TOO_LARGE and launches nothing
  *   plan_bitmap  device, ceil(vocab/32) words, bit v set iff token v is in P^plan; may be NULL when
