@@ -191,3 +191,31 @@ def test_small_tail_terms_are_not_lost_beside_a_dominant_logit(copies):
         assert np.max(np.abs(got["conf"][rows] - want["conf"])) <= 1e-4
         assert np.max(np.abs(got["ent"][rows] - want["ent"])) <= 3e-4
     ctx.close()
+
+
+@pytest.mark.parametrize("M", [24, 48, 200, 300])
+def test_hidden_states_written_just_before_the_call_are_the_ones_scored(M):
+    """Stream order: the scoring kernels fetch weights ahead of the work queued before them, never hidden states.
+    One buffer is overwritten on the stream right before every call, alternating between two sets of rows, with no
+    synchronisation in between; every call must see the rows written last (each kernel kind: streaming, swapped
+    paired, paired, swapped paired with two column groups)."""
+    V, D = 4096, 256
+    pos = np.arange(M)
+    st = synth.build_step("order", 4300, V, D, 64, [(pos, np.ones(M, np.uint8))], M, M, dict(tau_high=0.9, budget=4),
+                          amp_max=40.0)
+    w_bits, plan_ids = st.w_bits, st.plan_ids
+    sets = [st.h_bits, np.ascontiguousarray(st.h_bits[::-1])]          # the same rows in reverse order
+    want = [oscore.score(w_bits, s, plan_ids) for s in sets]
+    assert not np.array_equal(want[0]["tok"], want[1]["tok"])
+    ctx = make_ctx(w_bits, plan_ids, M)
+    src = [upload_bits(s) for s in sets]
+    h = torch.zeros_like(src[0])
+    outs = []
+    for i in range(12):
+        h.copy_(src[i % 2])                       # a kernel on the same stream, queued right before the call
+        outs.append(ctx.score(h))
+    torch.cuda.synchronize()
+    assert ctx.last_status() == 0
+    for i, out in enumerate(outs):
+        check_score(to_np(out), want[i % 2], V, plan_ids)
+    ctx.close()
