@@ -294,17 +294,29 @@ __device__ __forceinline__ void split_range(int units, int splits, int q, int *u
     *u1 = (int)((long long)units * (q + 1) / splits);
 }
 
+__device__ __forceinline__ int widest_range(int units, int splits) { return (units + splits - 1) / splits; }
+
 // Vocabulary tiles of a range of `range` granules starting at u0.  A short range (up to
 // kBalanceMaxTiles tiles) is cut into near-equal tiles: with full tiles plus a small ragged one, the
 // ragged tile's pipeline stages would hold too few bytes to keep HBM busy, and in the weight-streaming
 // regime that tile is a tenth of the block's work.  A long range keeps full tiles (one TMA box each).
+// `widest` (streaming kernel; 0 elsewhere) = the granules of the launch's widest range, ceil(units / splits): every
+// block then cuts its range into as many tiles as the widest one needs.  When HBM is saturated a block's share of it
+// follows the bytes it has in flight, i.e. its stage size; with V = 152064 a block of 64 granules (4 tiles of 16)
+// and its neighbour of 65 (5 tiles of 13) differ by a fifth in stage size, and the launch ended with the 65-granule
+// blocks 12 % after the others (measured per block: 181 us per launch, 173 with the same tile count everywhere).
+// The paired kernels lose more on the extra, narrower MMA tiles than they gain (measured), so they keep their own count.
 constexpr int kBalanceMaxTiles = 16;
 struct TileSplit {
     int u0, range, n_tiles, units_per_tile;
     bool balanced;
-    __device__ __forceinline__ TileSplit(int u0_, int u1_, int units_per_tile_)
-        : u0(u0_), range(u1_ - u0_), n_tiles((u1_ - u0_ + units_per_tile_ - 1) / units_per_tile_),
-          units_per_tile(units_per_tile_), balanced(n_tiles <= kBalanceMaxTiles) {}
+    __device__ __forceinline__ TileSplit(int u0_, int u1_, int units_per_tile_, int widest)
+        : u0(u0_), range(u1_ - u0_), n_tiles((max(u1_ - u0_, widest) + units_per_tile_ - 1) / units_per_tile_),
+          units_per_tile(units_per_tile_), balanced(n_tiles <= kBalanceMaxTiles)
+    {
+        if (!balanced) n_tiles = (range + units_per_tile - 1) / units_per_tile;
+        else if (n_tiles > range) n_tiles = max(range, 1);         // never an empty tile
+    }
     // first granule and number of granules of tile t
     __device__ __forceinline__ void tile(int t, int *tu0, int *tun) const
     {

@@ -69,7 +69,7 @@ pvf_score_gemm_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_con
     const int q = blockIdx.x / args.mb;
     int u0, u1;
     split_range(args.units, args.splits, q, &u0, &u1);
-    const TileSplit split(u0, u1, kUnitsPerTile);
+    const TileSplit split(u0, u1, kUnitsPerTile, 0);
     const int n_tiles = split.n_tiles;                                   // vocabulary tiles per sweep
     const int k_steps = (args.num_kb + kPanels - 1) / kPanels;
 

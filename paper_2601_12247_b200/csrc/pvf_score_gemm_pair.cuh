@@ -132,7 +132,7 @@ __device__ __forceinline__ int pair_prefetch_w(const ScoreArgs &args, const WMap
 {
     int s_tile, q, u0, u1;
     if (!pair_wave_work(args, pair, 0, &s_tile, &q, &u0, &u1)) return 0;
-    const TileSplit split(u0, u1, kPairUnitsPerTile);
+    const TileSplit split(u0, u1, kPairUnitsPerTile, 0);
     const uint64_t w_policy = w_evict_first_policy();
     int started = 0, ahead = 0;
     for (int tile = 0; tile < split.n_tiles && (started < kPairStages || ahead < kPairL2PrefetchSteps); ++tile) {
@@ -171,7 +171,7 @@ __device__ __forceinline__ void pair_produce(const ScoreArgs &args, const CUtens
         if (w > 0 && args.wave_sync) wave_boundary(args.wave_sync, (unsigned)w * gridDim.x);
         int s_tile, q, u0, u1;
         if (!pair_wave_work(args, pair, w, &s_tile, &q, &u0, &u1)) continue;
-        const TileSplit split(u0, u1, kPairUnitsPerTile);
+        const TileSplit split(u0, u1, kPairUnitsPerTile, 0);
         const int n_tiles = split.n_tiles;
         const int row0 = s_tile * 2 * kTileM + (int)rank * kTileM;          // this block's rows
         for (int tile = 0; tile < n_tiles && alive; ++tile) {
@@ -268,7 +268,7 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
             for (int w = 0; w < args.waves && alive; ++w) {
                 int s_tile, q, u0, u1;
                 if (!pair_wave_work(args, pair, w, &s_tile, &q, &u0, &u1)) continue;
-                const TileSplit split(u0, u1, kPairUnitsPerTile);
+                const TileSplit split(u0, u1, kPairUnitsPerTile, 0);
                 const int n_tiles = split.n_tiles;
                 for (int tile = 0; tile < n_tiles && alive; ++tile, ++tile_count) {
                     int tu0, tun;
@@ -311,7 +311,7 @@ pvf_score_gemm_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
         for (int w = 0; w < args.waves && alive; ++w) {
             int s_tile, q, u0, u1;
             if (!pair_wave_work(args, pair, w, &s_tile, &q, &u0, &u1)) continue;
-            const TileSplit split(u0, u1, kPairUnitsPerTile);
+            const TileSplit split(u0, u1, kPairUnitsPerTile, 0);
             const int n_tiles = split.n_tiles;
             const int row_base = s_tile * 2 * kTileM + (int)rank * kTileM;
             const int row = row_base + row_in_tile;

@@ -70,7 +70,7 @@ pvf_score_stream_kernel(const __grid_constant__ CUtensorMap tm_h, const __grid_c
     const int q = blockIdx.x;                                            // one vocabulary range per block
     int u0, u1;
     split_range(args.units, args.splits, q, &u0, &u1);
-    const TileSplit split(u0, u1, kStreamUnitsPerTile);
+    const TileSplit split(u0, u1, kStreamUnitsPerTile, widest_range(args.units, args.splits));
     const int n_tiles = split.n_tiles;
     const int n_cols = args.M <= 16 ? 16 : 32;                           // MMA N: scored rows, padded
     const int k_steps = args.num_kb;

@@ -221,7 +221,7 @@ pvf_score_swap_pair_kernel(const __grid_constant__ CUtensorMap tm_h, const __gri
     const int q = blockIdx.x >> 1;                                       // the pair's vocabulary range
     int u0, u1;
     split_range(args.units, args.splits, q, &u0, &u1);                   // granules of 32 entries
-    const TileSplit split(u0, u1, kPairUnitsPerTile);
+    const TileSplit split(u0, u1, kPairUnitsPerTile, 0);
     const int n_tiles = split.n_tiles;
     const int k_steps = args.num_kb;
 
