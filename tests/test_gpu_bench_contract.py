@@ -40,7 +40,7 @@ def test_default_workload_line():
     assert cfg["workload"] == "cfg1a" and cfg["draft_rows"] == 32 and "model" not in cfg
     # value = draft rows per second of the whole step
     assert d["value"] == pytest.approx(cfg["draft_rows"] / (d["ms_per_step"] * 1e-3), rel=1e-6)
-    assert d["gpu_launches"] == 4 * d["steps"]                      # 2 x projection (merge in its tail) + commit_select + verify
+    assert d["gpu_launches"] == 4 * d["steps"]                      # projection + draft kernel, projection + verify kernel
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["kernel"] == "pvf_score_stream_kernel"
     assert r["frac"] == pytest.approx(r["achieved"] / r["peak"], rel=1e-9)
@@ -55,7 +55,8 @@ def test_default_workload_line():
     for item in r["per_row_count"]:                               # the kernels' own clock: every launch of the region counted
         assert item["device_launches"] == d["steps"] * d["repeats"] and 500 < item["device_sm_mhz"] <= d["clocks"]["sm_max_mhz"] + 1
         assert item["device_sm_cycles"] == pytest.approx(item["device_kernel_us"] * item["device_sm_mhz"], rel=1e-6)
-        assert 0.8 * item["avg_launch_us"] < item["device_kernel_us"] <= 1.02 * item["avg_launch_us"]
+        # block 0's span starts when its wait returns: its first weight tiles were fetched before that
+        assert 0.75 * item["avg_launch_us"] < item["device_kernel_us"] <= 1.02 * item["avg_launch_us"]
     e = d["e2e"]
     assert e["unit"] == d["unit"] and e["h2d_bytes_per_step"] > 2 * 30 * 4096 * 2 and e["d2h_bytes_per_step"] > 0
     assert e["value"] < d["value"]                                   # host copies inside the timed region
