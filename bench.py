@@ -385,6 +385,16 @@ def run_workload(name, synth, binding, dev, world, rank, local_rank, peaks, step
     used = [(a, b, r) for a, b, r, blk in ev_pairs if event_every > 1 or blk == median_block]
     roof = roofline_of(used, ctx, V, D, peaks, clocks.get("sm_mhz"), event_every)
     roof["launches_timed_in"] = "the median block" if event_every == 1 else "all blocks"
+    # the same roofline for the step as a whole: what its two projection launches must move (or compute) against the
+    # step time, decision kernels and everything between the launches included
+    step_s = ms / steps * 1e-3
+    if roof["bound"] == "hbm":
+        step_alg = sum(2.0 * V * D + 2.0 * r * D + 13.0 * r + V / 8.0 for r in (M, Mv) if r > 0)
+        roof["step"] = dict(achieved=step_alg / step_s / 1e9, unit="GB/s", frac=step_alg / step_s / 1e9 / roof["peak"])
+    else:
+        step_alg = sum(2.0 * r * V * D for r in (M, Mv) if r > 0)
+        roof["step"] = dict(achieved=step_alg / step_s / 1e12, unit="TFLOP/s", frac=step_alg / step_s / 1e12 / roof["peak"],
+                            frac_sustained=step_alg / step_s / 1e12 / roof["peak_sustained"])
     # the kernels' own measurement over every launch of the timed region: run time and SM cycles of their first block
     for item in roof["per_row_count"]:
         c = device_clock.get(item["rows"])

@@ -49,6 +49,8 @@ def test_default_workload_line():
     # two projection launches per step cannot take longer than the step that contains them
     assert 2 * r["avg_launch_us"] * 1e-3 < d["ms_per_step"]
     launches_fit_the_step(r, d["ms_per_step"])
+    # the step as a whole (decision kernels and gaps included) against the same peak
+    assert r["step"]["unit"] == "GB/s" and 0.5 < r["step"]["frac"] <= r["frac"] * 1.0005
     assert r["timed_every_nth_step"] == 8 and d["repeats"] >= 20      # 24 steps of a third of a millisecond: many blocks
     assert d["clocks"]["samples"] >= 10 and d["clocks"]["sm_mhz"] > 0
     assert r["sm_cycles_per_launch"] == pytest.approx(r["avg_launch_us"] * d["clocks"]["sm_mhz"], rel=1e-9)
