@@ -532,7 +532,7 @@ def run_workload(name, synth, binding, dev, world, rank, local_rank, peaks, step
 
 
 def run_decode_loop(synth, binding, dev):
-    """BASELINE config 4: the synthetic decode loop (Algorithm 1) at batch 32, 256 tokens, blocks of 32, budget 4,
+    """Config 4: the synthetic decode loop (Algorithm 1) at batch 32, 256 tokens, blocks of 32, budget 4,
     PVF against confidence-threshold-only decoding (budget 0) on the same targets."""
     from paper_2601_12247_b200 import decode_loop
     V, D, B, L, S, K, seed = synth.LLADA_VOCAB, synth.LLADA_HIDDEN, 32, 256, 32, 4, 1004
@@ -587,8 +587,8 @@ def run_ours(args):
                 repeats=r["repeats"], clocks=r["clocks"], e2e=r["e2e"], gpu_launches=r["launches"], roofline=r["roofline"],
                 cpu_baseline=r["cpu_baseline"], parity=r["parity"], graph_replay=r["graph_replay"], status=r["status"])
 
-    # ---------------- beside the headline (single-GPU default run): the tensor-bound regime (BASELINE config 3) and
-    # the decode loop (BASELINE config 4), measured in the same process
+    # ---------------- beside the headline (single-GPU default run): the tensor-bound regime (config 3) and
+    # the decode loop (config 4), measured in the same process
     if world == 1 and args.workload == "cfg1a":
         if not args.no_tensor_regime:
             steps3 = 4
