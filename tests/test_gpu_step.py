@@ -129,6 +129,21 @@ def test_single_row_and_budget_zero(ctx):
     assert osel["n_drafts"].sum() == 0 and over["choice"].sum() == 0       # K = 0: threshold decoding only
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_single_sequence_writes_its_offsets_directly(ctx, seed):
+    """One sequence takes a path of its own in draft selection (no ticket, no packing): every budget, both routes,
+    lengths around a block of 256 threads, rows with and without the active flag."""
+    rng = np.random.default_rng(100 + seed)
+    max_len = [1, 7, 32, 64, 255, 256, 257, 600][seed]
+    c = random_case(rng, n_seq=1, max_len=max_len, K=[0, 1, 3, 4, 8, 16, 2, 5][seed], inactive=bool(seed % 2))
+    while c["M"] == 0:                                    # a sequence without rows says nothing here
+        c = random_case(rng, n_seq=1, max_len=max_len, K=c["K"], inactive=bool(seed % 2))
+    if seed % 3 == 0:
+        c["in_plan"][:] = 0                               # AR route (or none)
+    osel, over = run_step(ctx, c, rng=rng, flags=[0, 1, 2, 3][seed % 4])
+    assert osel["rem_off"][0] == 0 and osel["v_off"][0] == 0
+
+
 def test_argument_errors(ctx):
     prm = binding.make_params(0.9, 0.2, 0.65, 0.1, 64)      # budget above the context's limit
     seg = t_i32([0, 1])
