@@ -47,5 +47,18 @@ def test_host_step_equals_device_step(stress, pinned, bounce):
     assert np.array_equal(g["tok_v"][:Mv], dv["tok_v"]) and np.array_equal(g["conf_v"][:Mv], dv["conf_v"])
     for k in ("accept", "choice", "final_commit"):
         assert np.array_equal(g[k], dv[k]), k
+    # again and again on the same context: the results of every call are the call's own (nothing left over from
+    # the one before is taken for them)
+    for _ in range(4):
+        for v in hb.values():
+            v.zero_()
+        ctx.draft_step_host(prm, mk(binding.bf16_from_bits(st.h_bits, "cpu")), mk(torch.from_numpy(st.seg_off)),
+                            mk(torch.from_numpy(st.row_pos)), mk(torch.from_numpy(st.active)), hb)
+        for k in ("tok", "conf", "ent", "in_plan", "commit", "draft_rows", "n_drafts", "route", "rem_off", "v_off"):
+            assert np.array_equal(hb[k].numpy(), d[k]), k
+        ctx.verify_step_host(prm, mk(binding.bf16_from_bits(vp.hv_bits, "cpu")) if Mv else None, hb)
+        assert np.array_equal(hb["tok_v"].numpy()[:Mv], dv["tok_v"])
+        for k in ("accept", "choice", "final_commit"):
+            assert np.array_equal(hb[k].numpy(), dv[k]), k
     assert ctx.last_status() == 0
     ctx.close()
