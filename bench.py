@@ -41,13 +41,13 @@ UNIT = "positions/s"
 # waves (18 row tiles x 4 pairs each at the LLaDA shape) was captured at 3 waves; its traffic grows with the
 # number of waves, so larger launches scale the per-wave figure.
 NCU_TRAFFIC_PER_WAVE = {
-    "pvf_score_stream_kernel": 1.04032e9,
+    "pvf_score_stream_kernel": 1.04048e9,
     "pvf_score_gemm_kernel": None,
-    "pvf_score_gemm_pair_kernel": 1.04129e9,
-    "pvf_score_swap_pair_kernel": 1.04115e9,
+    "pvf_score_gemm_pair_kernel": 1.04131e9,
+    "pvf_score_swap_pair_kernel": 1.04149e9,
 }
-NCU_TRAFFIC_SWAP_WIDE = 1.0442e9          # the swapped paired kernel above 256 rows (two column groups)
-NCU_TRAFFIC_PAIR_MULTI_WAVE = 1.623e9     # the paired kernel, per wave, in launches of several waves
+NCU_TRAFFIC_SWAP_WIDE = 1.0423e9          # the swapped paired kernel above 256 rows (two column groups)
+NCU_TRAFFIC_PAIR_MULTI_WAVE = 1.674e9     # the paired kernel, per wave, in launches of several waves
 
 
 def load_peaks():
